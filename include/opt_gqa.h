@@ -1,0 +1,157 @@
+/*
+ * opt_gqa.h -- C ABI of the Opt-GQA attention library for NVIDIA B200 (sm_100a).
+ *
+ * Grouped-query attention in which the G = Hq / Hkv query heads of a group share
+ * one K/V head, K/V live in a paged (block-table) cache, and an ALiBi linear bias
+ * is added to the scores:
+ *
+ *     out[t,h,:] = sum_j softmax_j( scale * <q[t,h], k_j> - slope_h * (pos_t - j) ) * v_j
+ *
+ * with k_j, v_j the j-th cached token of the sequence, head h / G.
+ *
+ * Conventions common to every call
+ *  - Every pointer is a DEVICE pointer owned by the caller unless the argument is
+ *    documented as HOST.  The library allocates nothing and keeps no pointer after
+ *    the call returns; calls only enqueue work on `stream` (a cudaStream_t passed as
+ *    void*, NULL = the default stream) and return.  The caller keeps every buffer
+ *    alive until that work has finished.
+ *  - dtype: OPT_GQA_FP32 (0) or OPT_GQA_BF16 (1).  q, k_new/v_new, the cache and out
+ *    share it.  Slopes, scale, partials are always fp32.  All arithmetic is fp32;
+ *    results are rounded once (to nearest even) when stored.
+ *  - Cache layout: k_cache, v_cache are [num_blocks, Hkv, bs, D] row-major: one
+ *    (page, kv head) is one contiguous chunk of bs*D elements.
+ *  - Supported shapes: D in {64, 128}; bs in {16, 32}; G = Hq/Hkv in {1, 2, 4, 8}.
+ *  - Data pointers must be 16-byte aligned.
+ *  - Return value: 0 (OPT_GQA_OK) or a negative OPT_GQA_ERR_* code.  Argument checks
+ *    are done on the host before anything is enqueued; a failed check enqueues
+ *    nothing.  B = 0 or T = 0 returns OK without a launch.  There are no device
+ *    traps: a device-side wait that runs out records OPT_GQA_ERR_TIMEOUT in a status
+ *    word read by opt_gqa_device_status().
+ *  - Contract on index data (not checked on the device): context_lens[s] >= 0;
+ *    block_tables[s][i] is a valid page id for i < ceil(context_lens[s] / bs), and is
+ *    never read beyond that; slot_mapping entries are < num_blocks*bs and distinct
+ *    within one call (negative = skip the token).
+ *  - The tail of a sequence's last page and pages no sequence uses are never
+ *    interpreted: results do not depend on their contents (NaN bit patterns included).
+ */
+#ifndef OPT_GQA_H_
+#define OPT_GQA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OPT_GQA_FP32 0
+#define OPT_GQA_BF16 1
+
+#define OPT_GQA_OK 0
+#define OPT_GQA_ERR_NULL (-1)    /* a required pointer is NULL                            */
+#define OPT_GQA_ERR_SHAPE (-2)   /* unsupported or inconsistent sizes                     */
+#define OPT_GQA_ERR_DTYPE (-3)   /* dtype is neither OPT_GQA_FP32 nor OPT_GQA_BF16        */
+#define OPT_GQA_ERR_ALIGN (-4)   /* a data pointer is not 16-byte aligned                 */
+#define OPT_GQA_ERR_CUDA (-5)    /* the CUDA runtime refused the launch or a copy         */
+#define OPT_GQA_ERR_TIMEOUT (-6) /* a bounded device-side wait ran out (device status)    */
+
+/*
+ * Slot-mapped write of new tokens' K/V into the paged cache: Algorithm 1,
+ * "Reshape and store K, V into C_K, C_V" (same step in Algorithm 2; Eq. 2: the
+ * cached sequence is the earlier tokens followed by the new ones).
+ *
+ *   k_new, v_new  [T, Hkv, D]        rows of the T new tokens
+ *   k_cache, v_cache                 the pool, modified in place
+ *   slot_mapping  [T] int64          slot = page*bs + offset; token t goes to
+ *                                    cache[slot/bs][h][slot%bs][:] for every h;
+ *                                    a negative slot skips the token
+ * A bit-exact copy.  Call it before the attention call of the same step, on the
+ * same stream: context_lens passed to attention already counts these tokens.
+ */
+int opt_gqa_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                         const int64_t* slot_mapping, int T, int Hkv, int D, int bs,
+                         int64_t num_blocks, int dtype, void* stream);
+
+/*
+ * Decode attention over the paged cache, one query token per sequence at position
+ * n_s - 1: Algorithm 2, "Compute context attention with caches"; scores by Eq. 3
+ * (scaled dot product plus the ALiBi bias -slope_h*(n_s-1-j) of the "Integration
+ * and Optimization of ALiBi" paragraph), softmax by Eq. 4, weighted sum of V by
+ * Eq. 5; heads grouped as in "Query Grouping" / "Shared Key-Value" (query head h
+ * reads K/V head h / G).
+ *
+ *   out           [B, Hq, D]         written when partition_size == 0
+ *   q             [B, Hq, D]
+ *   block_tables  [B, max_blocks_per_seq] int32
+ *   context_lens  [B] int32          n_s, counts the current token; n_s == 0 gives
+ *                                    zero rows
+ *   alibi_slopes  [Hq] fp32, or NULL for no bias
+ *   partition_size  0: one CTA walks the whole sequence and writes out.
+ *                   P > 0 (a multiple of 16): the long-sequence split described
+ *                   before Eq. 1 -- CTA (s, kv head, p) attends to keys
+ *                   [pP, min((p+1)P, n_s)) and writes, for each head of the group,
+ *                   the normalised partial result and its log-sum-exp:
+ *                     partial_out [B, Hq, max_partitions, D] fp32
+ *                     partial_lse [B, Hq, max_partitions]    fp32 (natural log)
+ *                   for p < ceil(n_s / P); other entries are left untouched.  out
+ *                   is not written; follow with opt_gqa_paged_attention_reduce.
+ *                   max_partitions >= ceil(max_s n_s / P) is the caller's promise.
+ */
+int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* block_tables, int max_blocks_per_seq,
+                                   const int32_t* context_lens, const float* alibi_slopes, float scale,
+                                   int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                                   int partition_size, float* partial_out, float* partial_lse,
+                                   int max_partitions, int dtype, void* stream);
+
+/*
+ * Merge of the partitions' results (the paragraph before Eq. 1: "the output of
+ * each block is cached and then used" for the whole sequence):
+ *     out = sum_p e^{lse_p} o_p / sum_p e^{lse_p},   p < ceil(n_s / P)
+ * evaluated with the largest lse subtracted.  n_s == 0 gives zero rows.
+ * Arguments as written by opt_gqa_paged_attention_decode with the same
+ * partition_size and max_partitions.
+ */
+int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const float* partial_lse,
+                                   const int32_t* context_lens, int B, int Hq, int D, int partition_size,
+                                   int max_partitions, int dtype, void* stream);
+
+/*
+ * Multi-token (chunked-prefill) variant on tensor cores: the prompt branch of
+ * Algorithms 1 and 2 run over the paged cache with a causal mask plus the ALiBi
+ * bias ("Create ALiBi bias"; Eq. 3-5).  Sequence s contributes
+ * q_len_s = q_start_loc[s+1] - q_start_loc[s] new tokens whose K/V are already in
+ * the cache; new token i sits at position pos = n_s - q_len_s + i and attends to
+ * keys j <= pos with bias -slope_h*(pos - j).
+ *
+ *   out, q        [sum_s q_len_s, Hq, D]   (bf16 only)
+ *   q_start_loc   [B+1] int32              prefix sums of q_len_s, device memory
+ *   max_q_len     HOST value >= max_s q_len_s (sizes the grid)
+ */
+int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len,
+                                    const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                                    int max_blocks_per_seq, const int32_t* context_lens,
+                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D,
+                                    int bs, int64_t num_blocks, int dtype, void* stream);
+
+/*
+ * Bytes of fp32 scratch a split decode needs: partial_out followed by partial_lse,
+ * B*Hq*max_partitions*(D+1) floats.  (Workspace sizing for the partitioning step;
+ * pure host arithmetic.)  Returns 0 for non-positive arguments.
+ */
+size_t opt_gqa_workspace_bytes(int B, int Hq, int D, int max_partitions);
+
+/*
+ * Reads and clears the device status word of the current device: 0, or
+ * OPT_GQA_ERR_TIMEOUT if a bounded wait inside a kernel gave up since the last
+ * call.  Synchronises the device.  (Diagnostics; no counterpart in the paper.)
+ */
+int opt_gqa_device_status(void);
+
+/* Human-readable name of a status code.  Never NULL. */
+const char* opt_gqa_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OPT_GQA_H_ */

@@ -1,0 +1,134 @@
+"""ctypes binding of ``libopt_gqa.so``: argument marshalling only.
+
+Each function has the name of the C entry point it calls (without the
+``opt_gqa_`` prefix), takes CUDA torch tensors, passes their ``data_ptr()``
+and sizes straight through, and raises :class:`OptGqaError` on a non-zero
+status.  There is no fallback of any kind: if the shared library is missing
+or a tensor is not on a CUDA device the call fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libopt_gqa.so")
+
+FP32, BF16 = 0, 1
+_DTYPE_CODE = {torch.float32: FP32, torch.bfloat16: BF16}
+
+_c = ctypes
+_vp, _i, _i64, _f = _c.c_void_p, _c.c_int, _c.c_int64, _c.c_float
+
+SIGNATURES = {
+    "opt_gqa_cache_append": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i64, _i, _vp]),
+    "opt_gqa_paged_attention_decode": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
+                                            _i, _vp, _vp, _i, _i, _vp]),
+    "opt_gqa_paged_attention_reduce": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
+    "opt_gqa_paged_attention_prefill": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i,
+                                             _i, _i64, _i, _vp]),
+    "opt_gqa_workspace_bytes": (_c.c_size_t, [_i, _i, _i, _i]),
+    "opt_gqa_device_status": (_i, []),
+    "opt_gqa_status_string": (_c.c_char_p, [_i]),
+}
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+class OptGqaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+def load() -> ctypes.CDLL:
+    """Loads the shared library (built in-tree by ``paper_2505_02351_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2505_02351_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise OptGqaError(code, where)
+
+
+def status_string(code: int) -> str:
+    return load().opt_gqa_status_string(code).decode()
+
+
+def workspace_bytes(B: int, Hq: int, D: int, max_partitions: int) -> int:
+    return int(load().opt_gqa_workspace_bytes(B, Hq, D, max_partitions))
+
+
+def device_status() -> int:
+    return int(load().opt_gqa_device_status())
+
+
+def cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, stream=None) -> None:
+    T, Hkv, D = k_new.shape
+    num_blocks, _, bs, _ = k_cache.shape
+    assert slot_mapping.dtype == torch.int64
+    _check(load().opt_gqa_cache_append(_ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(slot_mapping),
+                                       T, Hkv, D, bs, num_blocks, _DTYPE_CODE[k_cache.dtype], _stream(stream)),
+           "opt_gqa_cache_append")
+
+
+def paged_attention_decode(out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
+                           partition_size: int = 0, partial_out=None, partial_lse=None, max_partitions: int = 0,
+                           stream=None) -> None:
+    B, Hq, D = q.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    assert block_tables.dtype == torch.int32 and context_lens.dtype == torch.int32
+    assert alibi_slopes is None or alibi_slopes.dtype == torch.float32
+    _check(load().opt_gqa_paged_attention_decode(
+        _ptr(out), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables), block_tables.shape[1],
+        _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size,
+        _ptr(partial_out), _ptr(partial_lse), max_partitions, _DTYPE_CODE[q.dtype], _stream(stream)),
+        "opt_gqa_paged_attention_decode")
+
+
+def paged_attention_reduce(out, partial_out, partial_lse, context_lens, partition_size: int, stream=None) -> None:
+    B, Hq, max_partitions, D = partial_out.shape
+    assert partial_out.dtype == torch.float32 and partial_lse.dtype == torch.float32
+    _check(load().opt_gqa_paged_attention_reduce(
+        _ptr(out), _ptr(partial_out), _ptr(partial_lse), _ptr(context_lens), B, Hq, D, partition_size,
+        max_partitions, _DTYPE_CODE[out.dtype], _stream(stream)), "opt_gqa_paged_attention_reduce")
+
+
+def paged_attention_prefill(out, q, q_start_loc, max_q_len: int, k_cache, v_cache, block_tables, context_lens,
+                            alibi_slopes, scale: float, stream=None) -> None:
+    T, Hq, D = q.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    B = context_lens.shape[0]
+    assert q_start_loc.dtype == torch.int32
+    _check(load().opt_gqa_paged_attention_prefill(
+        _ptr(out), _ptr(q), _ptr(q_start_loc), max_q_len, _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
+        block_tables.shape[1], _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks,
+        _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_prefill")

@@ -1,0 +1,144 @@
+// extern "C" boundary of the Opt-GQA library: host-side argument checks, then one
+// launcher per operation.  Nothing here allocates or keeps caller pointers.
+#include "common.cuh"
+
+namespace optgqa {
+
+// Written by kernels whose bounded waits give up; read and cleared by opt_gqa_device_status().
+__device__ int g_device_status = 0;
+
+static int* device_status_ptr() {
+    static int* ptrs[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        ptrs[dev] = static_cast<int*>(p);
+    }
+    return ptrs[dev];
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool dtype_ok(int dtype) { return dtype == OPT_GQA_FP32 || dtype == OPT_GQA_BF16; }
+static bool shape_ok(int Hq, int Hkv, int D, int bs) {
+    if (Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return false;
+    const int G = Hq / Hkv;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return false;
+    if (D != 64 && D != 128) return false;
+    if (bs != 16 && bs != 32) return false;
+    return true;
+}
+
+}  // namespace optgqa
+
+using namespace optgqa;
+
+extern "C" {
+
+int opt_gqa_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                         const int64_t* slot_mapping, int T, int Hkv, int D, int bs, int64_t num_blocks,
+                         int dtype, void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (T < 0 || Hkv <= 0 || (D != 64 && D != 128) || (bs != 16 && bs != 32) || num_blocks < 0) return OPT_GQA_ERR_SHAPE;
+    if (T == 0) return OPT_GQA_OK;
+    if (!k_new || !v_new || !k_cache || !v_cache || !slot_mapping) return OPT_GQA_ERR_NULL;
+    if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
+    return launch_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, T, Hkv, D, bs, dtype,
+                               static_cast<cudaStream_t>(stream));
+}
+
+int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* block_tables, int max_blocks_per_seq,
+                                   const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                   int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                                   float* partial_out, float* partial_lse, int max_partitions, int dtype,
+                                   void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0 || partition_size < 0 ||
+        partition_size % 16 != 0)
+        return OPT_GQA_ERR_SHAPE;
+    if (B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
+    if (B == 0) return OPT_GQA_OK;
+    if (!q || !k_cache || !v_cache || !block_tables || !context_lens) return OPT_GQA_ERR_NULL;
+    if (partition_size == 0) {
+        if (!out) return OPT_GQA_ERR_NULL;
+        if (!aligned16(out)) return OPT_GQA_ERR_ALIGN;
+    } else {
+        if (!partial_out || !partial_lse) return OPT_GQA_ERR_NULL;
+        if (max_partitions <= 0) return OPT_GQA_ERR_SHAPE;
+        if (!aligned16(partial_out)) return OPT_GQA_ERR_ALIGN;
+    }
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
+    int* status = device_status_ptr();
+    if (!status) return OPT_GQA_ERR_CUDA;
+    return launch_decode(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
+                         scale, B, Hq, Hkv, D, bs, partition_size, partial_out, partial_lse, max_partitions, dtype,
+                         status, static_cast<cudaStream_t>(stream));
+}
+
+int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const float* partial_lse,
+                                   const int32_t* context_lens, int B, int Hq, int D, int partition_size,
+                                   int max_partitions, int dtype, void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || Hq <= 0 || (D != 64 && D != 128) || partition_size <= 0 || partition_size % 16 != 0 ||
+        max_partitions <= 0)
+        return OPT_GQA_ERR_SHAPE;
+    if (B == 0) return OPT_GQA_OK;
+    if (!out || !partial_out || !partial_lse || !context_lens) return OPT_GQA_ERR_NULL;
+    if (!aligned16(out) || !aligned16(partial_out)) return OPT_GQA_ERR_ALIGN;
+    return launch_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size, max_partitions,
+                         dtype, static_cast<cudaStream_t>(stream));
+}
+
+int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len,
+                                    const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                                    int max_blocks_per_seq, const int32_t* context_lens,
+                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
+                                    int64_t num_blocks, int dtype, void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || max_q_len < 0 || !shape_ok(Hq, Hkv, D, bs) || D != 128 || max_blocks_per_seq < 0 || num_blocks < 0)
+        return OPT_GQA_ERR_SHAPE;
+    if (B == 0 || max_q_len == 0) return OPT_GQA_OK;
+    if (!out || !q || !q_start_loc || !k_cache || !v_cache || !block_tables || !context_lens) return OPT_GQA_ERR_NULL;
+    if (!aligned16(out) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
+    int* status = device_status_ptr();
+    if (!status) return OPT_GQA_ERR_CUDA;
+    return launch_prefill(out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables, max_blocks_per_seq,
+                          context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, status,
+                          static_cast<cudaStream_t>(stream));
+}
+
+size_t opt_gqa_workspace_bytes(int B, int Hq, int D, int max_partitions) {
+    if (B <= 0 || Hq <= 0 || D <= 0 || max_partitions <= 0) return 0;
+    return (size_t)B * (size_t)Hq * (size_t)max_partitions * (size_t)(D + 1) * sizeof(float);
+}
+
+int opt_gqa_device_status(void) {
+    int* p = device_status_ptr();
+    if (!p) return OPT_GQA_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, p, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    if (v != 0) {
+        int zero = 0;
+        if (cudaMemcpy(p, &zero, sizeof zero, cudaMemcpyHostToDevice) != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    }
+    return v;
+}
+
+const char* opt_gqa_status_string(int status) {
+    switch (status) {
+        case OPT_GQA_OK: return "ok";
+        case OPT_GQA_ERR_NULL: return "a required pointer is NULL";
+        case OPT_GQA_ERR_SHAPE: return "unsupported or inconsistent sizes";
+        case OPT_GQA_ERR_DTYPE: return "unsupported dtype";
+        case OPT_GQA_ERR_ALIGN: return "a data pointer is not 16-byte aligned";
+        case OPT_GQA_ERR_CUDA: return "CUDA runtime error";
+        case OPT_GQA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,126 @@
+// Shared device helpers of the Opt-GQA CUDA library (sm_100a): PTX wrappers for
+// mbarriers and bulk async copies, storage-type unpacking, launch plumbing.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "opt_gqa.h"
+
+namespace optgqa {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ----------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+
+// Makes freshly initialised barriers visible to the async proxy.
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// Orders earlier generic-proxy accesses to shared memory before later async-proxy ones.
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
+// Bounded wait: gives up after kSpinLimit polls, records the timeout and returns false.
+constexpr uint32_t kSpinLimit = 1u << 22;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    atomicExch(status, OPT_GQA_ERR_TIMEOUT);
+    return false;
+}
+
+// 1-D bulk copy global -> this CTA's shared memory, completion counted on `bar`.
+// dst, src 16-byte aligned; bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float lg2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Programmatic dependent launch: wait for the grid this one depends on / let dependents start.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ----------------------------------------------------------------------------- storage types
+// Two adjacent bf16 values packed in one 32-bit word -> (low element, high element) as fp32.
+__device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {
+    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+
+__device__ __forceinline__ uint32_t float2_to_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <typename T>
+struct Store;
+template <>
+struct Store<float> {
+    static constexpr int kDtype = OPT_GQA_FP32;
+};
+template <>
+struct Store<__nv_bfloat16> {
+    static constexpr int kDtype = OPT_GQA_BF16;
+};
+
+// ----------------------------------------------------------------------------- host-side launchers (one per .cu)
+int launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                        const int64_t* slot_mapping, int T, int Hkv, int D, int bs, int dtype,
+                        cudaStream_t stream);
+
+int launch_decode(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                  int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
+                  int B, int Hq, int Hkv, int D, int bs, int partition_size, float* partial_out,
+                  float* partial_lse, int max_partitions, int dtype, int* device_status, cudaStream_t stream);
+
+int launch_reduce(void* out, const float* partial_out, const float* partial_lse, const int32_t* context_lens,
+                  int B, int Hq, int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream);
+
+int launch_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len, const void* k_cache,
+                   const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
+                   const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
+                   int D, int bs, int* device_status, cudaStream_t stream);
+
+}  // namespace optgqa

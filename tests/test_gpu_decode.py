@@ -1,0 +1,121 @@
+"""Parity of the CUDA decode path (append -> decode -> reduce, through the C ABI) with the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_02351_b200 import binding
+from paper_2505_02351_b200 import workloads as W
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(wl, partition_size=None, **kw):
+    got, d = util.gpu_decode(wl, partition_size=partition_size, **kw)
+    want = util.oracle_attention(wl, **kw)
+    assert np.isfinite(got).all()
+    err = np.max(np.abs(got - want)) if got.size else 0.0
+    assert err <= util.TOL[wl.dtype], f"{wl.name}: max-abs error {err}"
+    return got, want, d
+
+
+def test_config1_tiny_fp32():
+    _check(W.make_config(1))
+    _check(W.make_config(1), partition_size=16)
+    _check(W.make_config(1), partition_size=48)
+
+
+def test_config1_poisoned_unused_slots():
+    _check(W.make_config(1, poison=True))
+    _check(W.make_config(1, poison=True), partition_size=32)
+
+
+def test_config2_bf16_llama7b_like():
+    _check(W.make_config(2))
+    _check(W.make_config(2, poison=True), partition_size=256)
+
+
+def test_config3_long_sequence_partitioned():
+    wl = W.make_config(3)
+    assert wl.partition_size == 512
+    _check(wl)
+
+
+def test_config4_ragged_large_batch_with_append():
+    wl = W.make_config(4, poison=True)
+    got, want, d = _check(wl, partition_size=512)
+    got1, _, _ = _check(wl, partition_size=0)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (4, 2), (8, 2), (8, 1)])
+@pytest.mark.parametrize("bs", [16, 32])
+def test_shape_matrix(dtype, D, Hq, Hkv, bs):
+    lens = [1, 15, 16, 17, 33, 100, 257, 0, 640]
+    wl = W.make_custom("m", dtype, Hq, Hkv, D, bs, lens, seed=D + Hq + bs, poison=True)
+    _check(wl)
+    _check(wl, partition_size=64)
+    _check(wl, partition_size=0, slopes=False)
+
+
+@pytest.mark.parametrize("P", [16, 48, 512, 4096])
+def test_any_partition_size_agrees_with_single_pass(P):
+    wl = W.make_custom("p", "bf16", 8, 2, 128, 16, [700, 33, 2049], seed=21)
+    _check(wl, partition_size=P)
+
+
+def test_partials_match_the_oracle_partials():
+    import oracle
+    wl = W.make_custom("p", "fp32", 4, 2, 64, 16, [130, 40, 77], seed=22)
+    got, d = util.gpu_decode(wl, partition_size=32)
+    a = util.oracle_inputs(wl)
+    maxP = d.partial_out.shape[2]
+    po, pl = oracle.partition_partials(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"], wl.scale, wl.dtype, 32, maxP)
+    gpo, gpl = d.partial_out.double().cpu().numpy(), d.partial_lse.double().cpu().numpy()
+    for s in range(wl.B):
+        np_s = (int(a["n"][s]) + 31) // 32
+        assert np.max(np.abs(gpo[s, :, :np_s] - po[s, :, :np_s])) < 1e-5
+        assert np.max(np.abs(gpl[s, :, :np_s] - pl[s, :, :np_s])) < 1e-5
+        assert np.isnan(gpo[s, :, np_s:]).all()          # entries past the sequence are left untouched
+
+
+def test_cache_append_is_bit_exact_and_touches_nothing_else():
+    import oracle
+    for dtype in ("fp32", "bf16"):
+        wl = W.make_custom("a", dtype, 8, 4, 128, 32, [70, 5, 300], q_lens=[7, 5, 33], seed=23)
+        d = util.DeviceWorkload(wl)
+        slots = wl.slot_mapping.clone()
+        slots[3] = -1
+        binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, slots.cuda())
+        torch.cuda.synchronize()
+        k = W.storage_numpy(wl.k_cache); v = W.storage_numpy(wl.v_cache)
+        oracle.cache_append(W.storage_numpy(wl.k_new), W.storage_numpy(wl.v_new), k, v, slots.numpy(), dtype)
+        assert np.array_equal(W.storage_numpy(d.k_cache), k)
+        assert np.array_equal(W.storage_numpy(d.v_cache), v)
+
+
+def test_page_permutation_leaves_the_result_bitwise_unchanged():
+    wl = W.make_custom("perm", "bf16", 8, 2, 128, 16, [300, 41], seed=24)
+    got, _ = util.gpu_decode(wl)
+    perm = torch.from_numpy(np.random.default_rng(1).permutation(wl.num_blocks))
+    k2 = torch.empty_like(wl.k_cache); v2 = torch.empty_like(wl.v_cache)
+    k2[perm] = wl.k_cache; v2[perm] = wl.v_cache
+    bt = wl.block_tables.long()
+    bt2 = torch.where(bt >= 0, perm[bt.clamp(min=0)], torch.full_like(bt, -1)).int()
+    slot2 = perm[wl.slot_mapping // wl.bs] * wl.bs + wl.slot_mapping % wl.bs
+    wl2 = W.Workload(**{**wl.__dict__, "k_cache": k2, "v_cache": v2, "block_tables": bt2, "slot_mapping": slot2})
+    got2, _ = util.gpu_decode(wl2)
+    assert np.array_equal(got, got2)
+
+
+def test_empty_batch_and_error_codes_on_device_pointers():
+    wl = W.make_config(1)
+    d = util.DeviceWorkload(wl)
+    empty = torch.empty((0, 4, 64), device="cuda")
+    binding.paged_attention_decode(empty, empty, d.k_cache, d.v_cache, d.block_tables[:0], d.context_lens[:0],
+                                   d.alibi_slopes, wl.scale)
+    with pytest.raises(binding.OptGqaError) as e:
+        binding.paged_attention_decode(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+                                       d.alibi_slopes, wl.scale, partition_size=20)
+    assert e.value.code == -2

@@ -1,0 +1,61 @@
+"""Helpers shared by the parity tests: run a workload through the CUDA library and through the oracle."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2505_02351_b200 import binding
+from paper_2505_02351_b200 import workloads as W
+
+TOL = {"fp32": 1e-5, "bf16": 2e-2}   # max-abs tolerance on attention outputs (fp32 accumulation)
+
+
+class DeviceWorkload:
+    """Device copies of a workload's tensors."""
+
+    def __init__(self, wl: W.Workload, device="cuda:0"):
+        self.wl = wl
+        dev = torch.device(device)
+        for name in ("q", "k_cache", "v_cache", "block_tables", "context_lens", "alibi_slopes", "k_new", "v_new",
+                     "slot_mapping"):
+            setattr(self, name, getattr(wl, name).to(dev))
+        self.q_start_loc = None if wl.q_start_loc is None else wl.q_start_loc.to(dev)
+        self.out = torch.full_like(self.q, float("nan"))
+
+
+def gpu_decode(wl: W.Workload, partition_size=None, append=True, slopes=True):
+    """append + decode (+ reduce) through the C ABI; returns (out float64 numpy, DeviceWorkload)."""
+    d = DeviceWorkload(wl)
+    P = wl.partition_size if partition_size is None else partition_size
+    if append:
+        binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
+    sl = d.alibi_slopes if slopes else None
+    if P > 0:
+        maxP = max(1, (int(wl.context_lens.max()) + P - 1) // P) if wl.B else 1
+        po = torch.full((wl.B, wl.Hq, maxP, wl.D), float("nan"), device="cuda:0", dtype=torch.float32)
+        pl = torch.full((wl.B, wl.Hq, maxP), float("nan"), device="cuda:0", dtype=torch.float32)
+        binding.paged_attention_decode(None, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, sl, wl.scale,
+                                       partition_size=P, partial_out=po, partial_lse=pl, max_partitions=maxP)
+        binding.paged_attention_reduce(d.out, po, pl, d.context_lens, P)
+        d.partial_out, d.partial_lse = po, pl
+    else:
+        binding.paged_attention_decode(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, sl, wl.scale)
+    torch.cuda.synchronize()
+    assert binding.device_status() == 0
+    return d.out.double().cpu().numpy(), d
+
+
+def oracle_inputs(wl: W.Workload, append=True):
+    k = W.storage_numpy(wl.k_cache)
+    v = W.storage_numpy(wl.v_cache)
+    if append:
+        oracle.cache_append(W.storage_numpy(wl.k_new), W.storage_numpy(wl.v_new), k, v, wl.slot_mapping.numpy(),
+                            wl.dtype)
+    return dict(q=W.storage_numpy(wl.q), k=k, v=v, bt=wl.block_tables.numpy(), n=wl.context_lens.numpy(),
+                slopes=wl.alibi_slopes.numpy().astype(np.float64),
+                qsl=None if wl.q_start_loc is None else wl.q_start_loc.numpy())
+
+
+def oracle_attention(wl: W.Workload, append=True, slopes=True):
+    a = oracle_inputs(wl, append)
+    return oracle.paged_attention(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"] if slopes else None, wl.scale,
+                                  wl.dtype, q_start_loc=a["qsl"])
