@@ -1,0 +1,496 @@
+#!/usr/bin/env python
+"""Benchmark of the Opt-GQA decode hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic input:
+cache_append of the step's new tokens -> paged GQA-ALiBi decode over context
+partitions -> log-sum-exp reduce.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 3] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run; the path shards by sequence with no
+data-path collective (every rank runs its own batch of the same shape), so the
+line reports weak scaling and the only communication is the timing reduction.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "paged GQA-ALiBi decode: achieved HBM TB/s vs peak; tokens/s per step"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+# Partition size used for workloads that do not fix one (the caller's choice under the C ABI).
+DEFAULT_PARTITION = {2: 256, 3: 512, 4: 512}
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised
+# under profiles/ (None until a capture of that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+# ----------------------------------------------------------------------------- distributed plumbing
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value: float, backend_device: str) -> float:
+    """MAX all-reduce of one float over the process group (identity when not initialised)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=backend_device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, backend_device: str) -> float:
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=backend_device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+# ----------------------------------------------------------------------------- clocks
+_REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+            0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU while the timed region runs (read-only NVML)."""
+
+    def __init__(self, device_index: int, period_s: float = 0.01):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples, self.reasons, self.sm_max = [], set(), None
+        self._halt = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _one(self):
+        nv = self._nv
+        self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+        try:
+            mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+        except Exception:
+            mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+        for bit, name in _REASONS.items():
+            if mask & bit:
+                self.reasons.add(name)
+
+    def run(self):
+        if self._h is None:
+            return
+        while not self._halt.is_set():
+            try:
+                self._one()
+            except Exception:
+                pass
+            self._halt.wait(self.period)
+
+    def stop(self) -> dict:
+        self._halt.set()
+        self.join(timeout=2.0)
+        if self._h is None or not self.samples:
+            return self._smi_fallback()
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.sm_max, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+    @staticmethod
+    def _smi_fallback() -> dict:
+        try:
+            out = subprocess.run(["nvidia-smi", "--query-gpu=clocks.sm,clocks.max.sm", "--format=csv,noheader,nounits"],
+                                 capture_output=True, text=True, timeout=10).stdout.strip().splitlines()[0]
+            a, b = [int(x) for x in out.split(",")]
+            return {"sm_mhz": a, "sm_max_mhz": b, "reasons": [], "samples": 1, "note": "one nvidia-smi sample after the run"}
+        except Exception:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+
+
+# ----------------------------------------------------------------------------- workload on the device
+class DeviceBatch:
+    """A workload resident in HBM, with `copies` distinct copies of the KV pool to rotate through."""
+
+    def __init__(self, wl, partition_size: int, copies: int, device):
+        import torch
+
+        from paper_2505_02351_b200 import binding
+
+        self.wl, self.P = wl, partition_size
+        self.dev = device
+        to = lambda t: t.to(device)
+        self.q, self.k_new, self.v_new = to(wl.q), to(wl.k_new), to(wl.v_new)
+        self.slots, self.tables, self.lens = to(wl.slot_mapping), to(wl.block_tables), to(wl.context_lens)
+        self.slopes = to(wl.alibi_slopes)
+        self.out = torch.zeros_like(self.q)
+        self.k_pools = [to(wl.k_cache)]
+        self.v_pools = [to(wl.v_cache)]
+        for _ in range(copies - 1):
+            self.k_pools.append(self.k_pools[0].clone())
+            self.v_pools.append(self.v_pools[0].clone())
+        self.maxP = max(1, (int(wl.context_lens.max()) + partition_size - 1) // partition_size) if partition_size else 1
+        ws = binding.workspace_bytes(wl.B, wl.Hq, wl.D, self.maxP) if partition_size else 0
+        self.workspace = torch.empty(max(ws, 16), dtype=torch.uint8, device=device)
+        self.partial_out = self.workspace[: wl.B * wl.Hq * self.maxP * wl.D * 4].view(torch.float32)
+        self.partial_lse = self.workspace[wl.B * wl.Hq * self.maxP * wl.D * 4: ws].view(torch.float32) if ws else None
+        self.lib = binding.load()
+        self.dt = binding.BF16 if wl.dtype == "bf16" else binding.FP32
+
+    # Pre-marshalled argument tuples: the timed loop then costs one foreign call per kernel.
+    def args_append(self, i, stream):
+        wl = self.wl
+        return (self.k_new.data_ptr(), self.v_new.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(),
+                self.slots.data_ptr(), wl.B, wl.Hkv, wl.D, wl.bs, wl.num_blocks, self.dt, stream)
+
+    def args_decode(self, i, stream):
+        wl = self.wl
+        return (self.out.data_ptr(), self.q.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(),
+                self.tables.data_ptr(), wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B,
+                wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, self.P,
+                self.partial_out.data_ptr() if self.P else None, self.partial_lse.data_ptr() if self.P else None,
+                self.maxP, self.dt, stream)
+
+    def args_reduce(self, stream):
+        wl = self.wl
+        return (self.out.data_ptr(), self.partial_out.data_ptr(), self.partial_lse.data_ptr(), self.lens.data_ptr(),
+                wl.B, wl.Hq, wl.D, self.P, self.maxP, self.dt, stream)
+
+    def args_step(self, i, stream):
+        wl = self.wl
+        return (self.out.data_ptr(), self.q.data_ptr(), self.k_new.data_ptr(), self.v_new.data_ptr(),
+                self.slots.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(), self.tables.data_ptr(),
+                wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D,
+                wl.bs, wl.num_blocks, self.P, self.workspace.data_ptr() if self.P else None, self.maxP, self.dt,
+                stream)
+
+    def algorithmic_bytes(self) -> int:
+        """Bytes one decode launch must move: every K and V element of every context once, q, out, table entries."""
+        wl = self.wl
+        es = 2 if wl.dtype == "bf16" else 4
+        n = wl.context_lens.long()
+        tables = int(((n + wl.bs - 1) // wl.bs).sum()) * 4
+        return wl.kv_bytes() + 2 * wl.B * wl.Hq * wl.D * es + tables
+
+
+def check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"{what} failed with status {rc}")
+
+
+def run_timed(batch: DeviceBatch, steps: int, warmup: int, per_kernel_events: bool):
+    """Warm-up, then `steps` steps timed with CUDA events on the launching stream.
+
+    Returns (total_ms, decode_ms_avg or None, launches).  Consecutive steps use different pool copies.
+    """
+    import torch
+
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+    lib, R, split = batch.lib, len(batch.k_pools), batch.P > 0
+    a_app = [batch.args_append(i, sh) for i in range(R)]
+    a_dec = [batch.args_decode(i, sh) for i in range(R)]
+    a_red = batch.args_reduce(sh) if split else None
+    f_app, f_dec, f_red = lib.opt_gqa_cache_append, lib.opt_gqa_paged_attention_decode, lib.opt_gqa_paged_attention_reduce
+
+    def step(i, ev=None):
+        check(f_app(*a_app[i % R]), "cache_append")
+        if ev is not None:
+            ev[0].record(stream)
+        check(f_dec(*a_dec[i % R]), "decode")
+        if ev is not None:
+            ev[1].record(stream)
+        if split:
+            check(f_red(*a_red), "reduce")
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)] \
+        if per_kernel_events else None
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    start.record(stream)
+    for i in range(steps):
+        step(warmup + i, evs[i] if evs else None)
+    end.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    total_ms = start.elapsed_time(end)
+    dec_ms = sum(a.elapsed_time(b) for a, b in evs) / steps if evs else None
+    return total_ms, dec_ms, steps * (3 if split else 2)
+
+
+def run_e2e(batch: DeviceBatch, steps: int, warmup: int):
+    """Steps through opt_gqa_decode_step_host: pinned host inputs copied in, result copied out, every step."""
+    import torch
+
+    from paper_2505_02351_b200 import binding
+
+    wl = batch.wl
+    pin = lambda t: t.contiguous().pin_memory()
+    hq, hk, hv = pin(wl.q), pin(wl.k_new), pin(wl.v_new)
+    hs, ht, hl = pin(wl.slot_mapping), pin(wl.block_tables), pin(wl.context_lens)
+    hout = torch.empty_like(wl.q).pin_memory()
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    staging = torch.empty(binding.step_staging_bytes(wl.B, wl.Hq, wl.Hkv, wl.D, wl.max_blocks, tdt), dtype=torch.uint8,
+                          device=batch.dev)
+    stream = torch.cuda.current_stream()
+    R = len(batch.k_pools)
+
+    def step(i):
+        binding.decode_step_host(hout, hq, hk, hv, hs, ht, hl, staging, batch.k_pools[i % R], batch.v_pools[i % R],
+                                 batch.slopes, wl.scale, partition_size=batch.P,
+                                 workspace=batch.workspace if batch.P else None, max_partitions=batch.maxP)
+        stream.synchronize()          # the caller reads out_host after every step
+
+    for i in range(warmup):
+        step(i)
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(steps):
+        step(warmup + i)
+    dt = time.perf_counter() - t0
+    barrier()
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hs, ht, hl))
+    d2h = hout.numel() * hout.element_size()
+    return dt, h2d, d2h, hout
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_step_fn(wl):
+    """Returns (fn(units) -> seconds, total_units): the oracle's append + decode on the first `units` sequences."""
+    import numpy as np
+
+    import oracle
+    from paper_2505_02351_b200 import workloads as W
+
+    k, v = W.storage_numpy(wl.k_cache), W.storage_numpy(wl.v_cache)
+    q, kn, vn = W.storage_numpy(wl.q), W.storage_numpy(wl.k_new), W.storage_numpy(wl.v_new)
+    bt, n, slots = wl.block_tables.numpy(), wl.context_lens.numpy(), wl.slot_mapping.numpy()
+    slopes = wl.alibi_slopes.numpy().astype(np.float64)
+
+    def fn(units: int) -> float:
+        t0 = time.perf_counter()
+        oracle.cache_append(kn[:units], vn[:units], k, v, slots[:units], wl.dtype)
+        oracle.paged_attention(q[:units], k, v, bt[:units], n[:units], slopes, wl.scale, wl.dtype)
+        return time.perf_counter() - t0
+
+    return fn, wl.B
+
+
+def omp_threads() -> int:
+    v = os.environ.get("OMP_NUM_THREADS")
+    if v and v.isdigit():
+        return int(v)
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(wl, budget_s: float = 12.0) -> dict:
+    fn, B = oracle_step_fn(wl)
+    t1 = fn(B)
+    reps = int(min(20, max(1, math.floor(budget_s / max(t1, 1e-3)) - 1)))
+    times = [t1] + [fn(B) for _ in range(reps - 1)] if reps > 1 else [t1]
+    best = min(times)
+    return {"value": B / best, "unit": UNIT, "cores": omp_threads(), "kind": "oracle",
+            "sample": f"fp64 C oracle (append + decode) on the full batch of {B} sequences, best of {len(times)} passes, "
+                      f"{best:.3f} s per pass"}
+
+
+def run_reference(args, wl, rank: int):
+    """--impl reference: the oracle as it stands, on the host cores; each step a bounded sample."""
+    fn, B = oracle_step_fn(wl)
+    steps = args.steps if args.steps is not None else 5
+    warmup = args.warmup if args.warmup is not None else 1
+    t_full = fn(B)
+    budget = 150.0
+    units = int(max(1, min(B, math.floor(B * budget / max(t_full * (steps + warmup), 1e-6)))))
+    for _ in range(warmup):
+        fn(units)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        fn(units)
+    dt = time.perf_counter() - t0
+    value = units * steps / dt
+    sample = f"fp64 C oracle (append + decode) on the first {units} of {B} sequences per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.B, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.D,
+                   "block_size": wl.bs, "storage_dtype": wl.dtype, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": omp_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- main
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", type=int, default=3, choices=[2, 3, 4],
+                    help="named workload (1-based): 3 = long-sequence decode, the headline")
+    ap.add_argument("--partition", type=int, default=None, help="context partition size (default: the workload's)")
+    ap.add_argument("--copies", type=int, default=4, help="distinct KV pool copies rotated between steps")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the short side measurements of the other workloads")
+    args = ap.parse_args()
+    rank, local_rank, world = dist_env()
+
+    from paper_2505_02351_b200 import workloads as W
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        wl = W.make_config(args.config)
+        run_reference(args, wl, rank)
+        return
+
+    import torch
+
+    from paper_2505_02351_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    binding.load()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    steps = args.steps if args.steps is not None else 4000
+    warmup = max(3, args.warmup if args.warmup is not None else 50)
+
+    wl = W.make_config(args.config, seed_offset=1000 * rank)
+    P = args.partition if args.partition is not None else (wl.partition_size or DEFAULT_PARTITION[args.config])
+    batch = DeviceBatch(wl, P, args.copies, dev)
+    pool_bytes = sum(t.numel() * t.element_size() for t in batch.k_pools + batch.v_pools)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    total_ms, dec_ms, launches = run_timed(batch, steps, warmup, per_kernel_events=True)
+    clocks = sampler.stop()
+    status = binding.device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status}: {binding.status_string(status)}")
+    total_ms = max_over_ranks(total_ms, str(dev))
+    tokens_all = sum_over_ranks(float(wl.B), str(dev))
+    value = tokens_all * steps / (total_ms * 1e-3)
+
+    e2e_steps = min(steps, 500)
+    if args.no_e2e:
+        e2e_s, h2d, d2h = float("nan"), 0, 0
+    else:
+        e2e_s, h2d, d2h, _ = run_e2e(batch, e2e_steps, 10)
+        e2e_s = max_over_ranks(e2e_s, str(dev))
+    e2e_value = tokens_all * e2e_steps / e2e_s
+
+    peak, peak_kind = measured_peak()
+    alg = batch.algorithmic_bytes()
+    achieved = alg / (dec_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                "algorithmic_bytes_per_launch": alg, "kernel_us": dec_ms * 1e3,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "batch_per_gpu": wl.B, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.D,
+                   "block_size": wl.bs, "storage_dtype": wl.dtype, "partition_size": P,
+                   "context_tokens_per_gpu": int(wl.context_lens.sum()), "parallelism": f"dp{world} (by sequence, no collective)",
+                   "step": "cache_append + decode + reduce",
+                   "l2": f"{args.copies} distinct KV pool copies ({pool_bytes / 1e9:.2f} GB) rotated between steps; "
+                         f"each step reads {wl.kv_bytes() / 1e6:.0f} MB (> 126 MB L2)"},
+        "hbm_tbs_step": alg * tokens_all / wl.B / (total_ms / steps * 1e-3) / 1e12,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "api": "opt_gqa_decode_step_host (pinned host q/k_new/v_new/slots/tables/lens in, out back, sync per step)"},
+        "gpu_launches": launches,
+        "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1 and not args.no_extra:
+        extra = {}
+        for cfg in (2, 4):
+            if cfg == args.config:
+                continue
+            w2 = W.make_config(cfg)
+            b2 = DeviceBatch(w2, w2.partition_size or DEFAULT_PARTITION[cfg], args.copies, dev)
+            t_ms, d_ms, _ = run_timed(b2, 1000, 20, per_kernel_events=True)
+            a2 = b2.algorithmic_bytes()
+            extra[w2.name] = {"tokens_per_s": w2.B * 1000 / (t_ms * 1e-3), "ms_per_step": t_ms / 1000,
+                              "decode_us": d_ms * 1e3, "decode_GBs": a2 / (d_ms * 1e-3) / 1e9,
+                              "frac_of_peak": a2 / (d_ms * 1e-3) / 1e9 / peak, "partition_size": b2.P}
+            del b2, w2
+            torch.cuda.empty_cache()
+        line["other_workloads"] = extra
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

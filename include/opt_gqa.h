@@ -105,8 +105,8 @@ int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache
                                    int max_partitions, int dtype, void* stream);
 
 /*
- * Merge of the partitions' results (the paragraph before Eq. 1: "the output of
- * each block is cached and then used" for the whole sequence):
+ * Merge of the partitions' results (the paragraph before Eq. 1: each partition's
+ * output is kept and then combined into the result for the whole sequence):
  *     out = sum_p e^{lse_p} o_p / sum_p e^{lse_p},   p < ceil(n_s / P)
  * evaluated with the largest lse subtracted.  n_s == 0 gives zero rows.
  * Arguments as written by opt_gqa_paged_attention_decode with the same
@@ -133,6 +133,44 @@ int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_s
                                     int max_blocks_per_seq, const int32_t* context_lens,
                                     const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D,
                                     int bs, int64_t num_blocks, int dtype, void* stream);
+
+/*
+ * One decode step of the attention layer, Algorithm 2 from "Store reshaped K, V
+ * into C_K, C_V" to "Compute context attention with caches": cache_append of the
+ * B new tokens (k_new, v_new [B, Hkv, D], slot_mapping [B]), then decode, then --
+ * when partition_size > 0 -- the reduce, all enqueued on `stream` by one call.
+ * workspace: opt_gqa_workspace_bytes(B, Hq, D, max_partitions) bytes of device
+ * memory (partial_out followed by partial_lse); may be NULL when partition_size
+ * is 0.  Other arguments as in the three calls it chains.  out [B, Hq, D] is
+ * always written.
+ */
+int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,
+                        const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,
+                        int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,
+                        float scale, int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                        int partition_size, void* workspace, int max_partitions, int dtype, void* stream);
+
+/*
+ * The same step for a caller whose per-step tensors live in HOST memory (pinned,
+ * for the copies to be asynchronous): out_host, q_host, k_new_host, v_new_host,
+ * slot_mapping_host, block_tables_host, context_lens_host are HOST pointers with
+ * the shapes above.  They are copied to `staging` (device memory of
+ * opt_gqa_step_staging_bytes(...) bytes, 256-byte aligned) on `stream`, the step
+ * runs there, and out is copied back to out_host; the call returns once everything
+ * is enqueued, so synchronise `stream` before reading out_host or reusing the host
+ * buffers.  The cache, alibi_slopes and workspace stay DEVICE pointers: the cache
+ * is state that persists between steps.  (Convenience wrapper around the step; the
+ * transfers are the "Reshape Q, K, V" hand-over of Algorithm 2's inputs.)
+ */
+int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_new_host, const void* v_new_host,
+                             const int64_t* slot_mapping_host, const int32_t* block_tables_host,
+                             const int32_t* context_lens_host, void* staging, void* k_cache, void* v_cache,
+                             int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
+                             int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
+                             int max_partitions, int dtype, void* stream);
+
+/* Device bytes opt_gqa_decode_step_host needs in `staging`.  Host arithmetic; 0 for bad arguments. */
+size_t opt_gqa_step_staging_bytes(int B, int Hq, int Hkv, int D, int max_blocks_per_seq, int dtype);
 
 /*
  * Bytes of fp32 scratch a split decode needs: partial_out followed by partial_lse,

@@ -195,8 +195,9 @@ int oracle_partition_partials(double* partial_out, double* partial_lse, const vo
 }
 
 /*
- * Combining the partitions ("the output of each block is cached and then
- * used ..."): softmax over the whole context splits exactly as
+ * Combining the partitions (the paragraph before Eq. 1 keeps each partition's
+ * output and feeds it into the sequence's result): softmax over the whole
+ * context splits exactly as
  *   out = sum_p e^{lse_p} o_p / sum_p e^{lse_p},  p < ceil(n_s / P),
  * evaluated with the largest lse subtracted.  n_s = 0 gives zeros.
  */

@@ -30,6 +30,11 @@ SIGNATURES = {
     "opt_gqa_paged_attention_reduce": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_prefill": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i,
                                              _i, _i64, _i, _vp]),
+    "opt_gqa_decode_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
+                                 _i, _vp, _i, _i, _vp]),
+    "opt_gqa_decode_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _f, _i, _i, _i, _i,
+                                      _i, _i64, _i, _vp, _i, _i, _vp]),
+    "opt_gqa_step_staging_bytes": (_c.c_size_t, [_i, _i, _i, _i, _i, _i]),
     "opt_gqa_workspace_bytes": (_c.c_size_t, [_i, _i, _i, _i]),
     "opt_gqa_device_status": (_i, []),
     "opt_gqa_status_string": (_c.c_char_p, [_i]),
@@ -132,3 +137,38 @@ def paged_attention_prefill(out, q, q_start_loc, max_q_len: int, k_cache, v_cach
         _ptr(out), _ptr(q), _ptr(q_start_loc), max_q_len, _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
         block_tables.shape[1], _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks,
         _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_prefill")
+
+
+def step_staging_bytes(B: int, Hq: int, Hkv: int, D: int, max_blocks_per_seq: int, dtype: torch.dtype) -> int:
+    return int(load().opt_gqa_step_staging_bytes(B, Hq, Hkv, D, max_blocks_per_seq, _DTYPE_CODE[dtype]))
+
+
+def decode_step(out, q, k_new, v_new, slot_mapping, k_cache, v_cache, block_tables, context_lens, alibi_slopes,
+                scale: float, partition_size: int = 0, workspace=None, max_partitions: int = 0, stream=None) -> None:
+    B, Hq, D = q.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    _check(load().opt_gqa_decode_step(
+        _ptr(out), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(slot_mapping), _ptr(k_cache), _ptr(v_cache),
+        _ptr(block_tables), block_tables.shape[1], _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs,
+        num_blocks, partition_size, _ptr(workspace), max_partitions, _DTYPE_CODE[q.dtype], _stream(stream)),
+        "opt_gqa_decode_step")
+
+
+def _host_ptr(t: torch.Tensor) -> int:
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous host tensor")
+    return t.data_ptr()
+
+
+def decode_step_host(out_host, q_host, k_new_host, v_new_host, slot_mapping_host, block_tables_host,
+                     context_lens_host, staging, k_cache, v_cache, alibi_slopes, scale: float,
+                     partition_size: int = 0, workspace=None, max_partitions: int = 0, stream=None) -> None:
+    """Host tensors (pinned) in and out; cache, slopes, staging and workspace on the device.  Does not synchronise."""
+    B, Hq, D = q_host.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    _check(load().opt_gqa_decode_step_host(
+        _host_ptr(out_host), _host_ptr(q_host), _host_ptr(k_new_host), _host_ptr(v_new_host),
+        _host_ptr(slot_mapping_host), _host_ptr(block_tables_host), _host_ptr(context_lens_host), _ptr(staging),
+        _ptr(k_cache), _ptr(v_cache), block_tables_host.shape[1], _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs,
+        num_blocks, partition_size, _ptr(workspace), max_partitions, _DTYPE_CODE[q_host.dtype], _stream(stream)),
+        "opt_gqa_decode_step_host")

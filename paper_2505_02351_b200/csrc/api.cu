@@ -111,6 +111,92 @@ int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_s
                           static_cast<cudaStream_t>(stream));
 }
 
+int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,
+                        const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,
+                        int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,
+                        float scale, int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                        int partition_size, void* workspace, int max_partitions, int dtype, void* stream) {
+    if (!out) return B == 0 ? OPT_GQA_OK : OPT_GQA_ERR_NULL;
+    if (partition_size > 0 && !workspace && B > 0) return OPT_GQA_ERR_NULL;
+    int rc = opt_gqa_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, B, Hkv, D, bs, num_blocks, dtype,
+                                  stream);
+    if (rc != OPT_GQA_OK) return rc;
+    float* partial_out = static_cast<float*>(workspace);
+    float* partial_lse =
+        partial_out ? partial_out + (size_t)(B > 0 ? B : 0) * Hq * (max_partitions > 0 ? max_partitions : 0) * D
+                    : nullptr;
+    rc = opt_gqa_paged_attention_decode(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+                                        alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size,
+                                        partial_out, partial_lse, max_partitions, dtype, stream);
+    if (rc != OPT_GQA_OK || partition_size == 0) return rc;
+    return opt_gqa_paged_attention_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size,
+                                          max_partitions, dtype, stream);
+}
+
+namespace {
+struct StagingLayout {
+    size_t q, k_new, v_new, out, slots, tables, lens, total;
+};
+size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
+bool staging_layout(int B, int Hq, int Hkv, int D, int max_blocks, int dtype, StagingLayout* L) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || max_blocks < 0 || !dtype_ok(dtype)) return false;
+    const size_t es = dtype == OPT_GQA_FP32 ? 4 : 2;
+    size_t off = 0;
+    L->q = off, off += round256((size_t)B * Hq * D * es);
+    L->k_new = off, off += round256((size_t)B * Hkv * D * es);
+    L->v_new = off, off += round256((size_t)B * Hkv * D * es);
+    L->out = off, off += round256((size_t)B * Hq * D * es);
+    L->slots = off, off += round256((size_t)B * sizeof(int64_t));
+    L->tables = off, off += round256((size_t)B * max_blocks * sizeof(int32_t));
+    L->lens = off, off += round256((size_t)B * sizeof(int32_t));
+    L->total = off;
+    return true;
+}
+}  // namespace
+
+size_t opt_gqa_step_staging_bytes(int B, int Hq, int Hkv, int D, int max_blocks_per_seq, int dtype) {
+    StagingLayout L;
+    return staging_layout(B, Hq, Hkv, D, max_blocks_per_seq, dtype, &L) ? L.total : 0;
+}
+
+int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_new_host, const void* v_new_host,
+                             const int64_t* slot_mapping_host, const int32_t* block_tables_host,
+                             const int32_t* context_lens_host, void* staging, void* k_cache, void* v_cache,
+                             int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
+                             int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
+                             int max_partitions, int dtype, void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0) return OPT_GQA_ERR_SHAPE;
+    if (B == 0) return OPT_GQA_OK;
+    if (!out_host || !q_host || !k_new_host || !v_new_host || !slot_mapping_host || !block_tables_host ||
+        !context_lens_host || !staging)
+        return OPT_GQA_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(staging) & 255u) != 0) return OPT_GQA_ERR_ALIGN;
+    StagingLayout L;
+    if (!staging_layout(B, Hq, Hkv, D, max_blocks_per_seq, dtype, &L)) return OPT_GQA_ERR_SHAPE;
+    const size_t es = dtype == OPT_GQA_FP32 ? 4 : 2;
+    char* st = static_cast<char*>(staging);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const size_t qb = (size_t)B * Hq * D * es, kb = (size_t)B * Hkv * D * es;
+    bool ok = true;
+    ok &= cudaMemcpyAsync(st + L.q, q_host, qb, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + L.k_new, k_new_host, kb, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + L.v_new, v_new_host, kb, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + L.slots, slot_mapping_host, (size_t)B * 8, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + L.tables, block_tables_host, (size_t)B * max_blocks_per_seq * 4,
+                          cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + L.lens, context_lens_host, (size_t)B * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    if (!ok) return OPT_GQA_ERR_CUDA;
+    int rc = opt_gqa_decode_step(st + L.out, st + L.q, st + L.k_new, st + L.v_new,
+                                 reinterpret_cast<const int64_t*>(st + L.slots), k_cache, v_cache,
+                                 reinterpret_cast<const int32_t*>(st + L.tables), max_blocks_per_seq,
+                                 reinterpret_cast<const int32_t*>(st + L.lens), alibi_slopes, scale, B, Hq, Hkv, D,
+                                 bs, num_blocks, partition_size, workspace, max_partitions, dtype, stream);
+    if (rc != OPT_GQA_OK) return rc;
+    if (cudaMemcpyAsync(out_host, st + L.out, qb, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    return OPT_GQA_OK;
+}
+
 size_t opt_gqa_workspace_bytes(int B, int Hq, int D, int max_partitions) {
     if (B <= 0 || Hq <= 0 || D <= 0 || max_partitions <= 0) return 0;
     return (size_t)B * (size_t)Hq * (size_t)max_partitions * (size_t)(D + 1) * sizeof(float);

@@ -188,10 +188,10 @@ def config_lengths(cfg: int, shrink: int = 1):
     raise ValueError(cfg)
 
 
-def make_config(cfg: int, poison: bool = False, shrink: int = 1) -> Workload:
-    """The five named workloads (1-based), seeds 0..4."""
+def make_config(cfg: int, poison: bool = False, shrink: int = 1, seed_offset: int = 0) -> Workload:
+    """The five named workloads (1-based), seeds 0..4 (``seed_offset`` gives other ranks their own values)."""
     n, ql = config_lengths(cfg, shrink)
-    seed = cfg - 1
+    seed = cfg - 1 + seed_offset
     shape = {
         1: dict(dtype="fp32", Hq=4, Hkv=2, D=64, bs=16, partition_size=0),
         2: dict(dtype="bf16", Hq=32, Hkv=8, D=128, bs=16, partition_size=0),
