@@ -105,6 +105,21 @@ int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache
                                    int max_partitions, int dtype, void* stream);
 
 /*
+ * The same operation, arguments and results as opt_gqa_paged_attention_decode, forced
+ * onto the CUDA-core kernel (16 lanes per token row, warp-shuffle reduce-scatter of the
+ * G partial dot products, packed fp32 FMAs).  opt_gqa_paged_attention_decode uses this
+ * kernel for fp32 caches and a tensor-core tile kernel (the query group as the rows of
+ * m16n8k16 tiles) for bf16 caches; this entry point keeps the CUDA-core form of Eq. 3-5
+ * reachable for bf16 as well, for comparison and as a cross-check.
+ */
+int opt_gqa_paged_attention_decode_simt(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                        const int32_t* block_tables, int max_blocks_per_seq,
+                                        const int32_t* context_lens, const float* alibi_slopes, float scale,
+                                        int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                                        int partition_size, float* partial_out, float* partial_lse,
+                                        int max_partitions, int dtype, void* stream);
+
+/*
  * Merge of the partitions' results (the paragraph before Eq. 1: each partition's
  * output is kept and then combined into the result for the whole sequence):
  *     out = sum_p e^{lse_p} o_p / sum_p e^{lse_p},   p < ceil(n_s / P)

@@ -27,6 +27,8 @@ SIGNATURES = {
     "opt_gqa_cache_append": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i64, _i, _vp]),
     "opt_gqa_paged_attention_decode": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                             _i, _vp, _vp, _i, _i, _vp]),
+    "opt_gqa_paged_attention_decode_simt": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
+                                                 _i, _vp, _vp, _i, _i, _vp]),
     "opt_gqa_paged_attention_reduce": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_prefill": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i,
                                              _i, _i64, _i, _vp]),
@@ -105,18 +107,30 @@ def cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, stream=None) -> N
            "opt_gqa_cache_append")
 
 
-def paged_attention_decode(out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
-                           partition_size: int = 0, partial_out=None, partial_lse=None, max_partitions: int = 0,
-                           stream=None) -> None:
+def _decode(entry: str, out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale, partition_size,
+            partial_out, partial_lse, max_partitions, stream) -> None:
     B, Hq, D = q.shape
     num_blocks, Hkv, bs, _ = k_cache.shape
     assert block_tables.dtype == torch.int32 and context_lens.dtype == torch.int32
     assert alibi_slopes is None or alibi_slopes.dtype == torch.float32
-    _check(load().opt_gqa_paged_attention_decode(
+    _check(getattr(load(), entry)(
         _ptr(out), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables), block_tables.shape[1],
         _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size,
-        _ptr(partial_out), _ptr(partial_lse), max_partitions, _DTYPE_CODE[q.dtype], _stream(stream)),
-        "opt_gqa_paged_attention_decode")
+        _ptr(partial_out), _ptr(partial_lse), max_partitions, _DTYPE_CODE[q.dtype], _stream(stream)), entry)
+
+
+def paged_attention_decode(out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
+                           partition_size: int = 0, partial_out=None, partial_lse=None, max_partitions: int = 0,
+                           stream=None) -> None:
+    _decode("opt_gqa_paged_attention_decode", out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes,
+            scale, partition_size, partial_out, partial_lse, max_partitions, stream)
+
+
+def paged_attention_decode_simt(out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
+                                partition_size: int = 0, partial_out=None, partial_lse=None,
+                                max_partitions: int = 0, stream=None) -> None:
+    _decode("opt_gqa_paged_attention_decode_simt", out, q, k_cache, v_cache, block_tables, context_lens,
+            alibi_slopes, scale, partition_size, partial_out, partial_lse, max_partitions, stream)
 
 
 def paged_attention_reduce(out, partial_out, partial_lse, context_lens, partition_size: int, stream=None) -> None:

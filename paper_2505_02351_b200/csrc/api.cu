@@ -49,12 +49,11 @@ int opt_gqa_cache_append(const void* k_new, const void* v_new, void* k_cache, vo
                                static_cast<cudaStream_t>(stream));
 }
 
-int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache, const void* v_cache,
-                                   const int32_t* block_tables, int max_blocks_per_seq,
-                                   const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
-                                   int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                                   float* partial_out, float* partial_lse, int max_partitions, int dtype,
-                                   void* stream) {
+static int decode_checked(bool allow_tensor_cores, void* out, const void* q, const void* k_cache, const void* v_cache,
+                          const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
+                          const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
+                          int64_t num_blocks, int partition_size, float* partial_out, float* partial_lse,
+                          int max_partitions, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0 || partition_size < 0 ||
         partition_size % 16 != 0)
@@ -62,20 +61,48 @@ int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache
     if (B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
     if (B == 0) return OPT_GQA_OK;
     if (!q || !k_cache || !v_cache || !block_tables || !context_lens) return OPT_GQA_ERR_NULL;
+    if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
     if (partition_size == 0) {
         if (!out) return OPT_GQA_ERR_NULL;
         if (!aligned16(out)) return OPT_GQA_ERR_ALIGN;
     } else {
         if (!partial_out || !partial_lse) return OPT_GQA_ERR_NULL;
-        if (max_partitions <= 0) return OPT_GQA_ERR_SHAPE;
+        if (max_partitions <= 0 || max_partitions > 65535) return OPT_GQA_ERR_SHAPE;
         if (!aligned16(partial_out)) return OPT_GQA_ERR_ALIGN;
     }
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (allow_tensor_cores && dtype == OPT_GQA_BF16)
+        return launch_decode_tc(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+                                alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
+                                partial_lse, max_partitions, status, cs);
     return launch_decode(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
                          scale, B, Hq, Hkv, D, bs, partition_size, partial_out, partial_lse, max_partitions, dtype,
-                         status, static_cast<cudaStream_t>(stream));
+                         status, cs);
+}
+
+int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* block_tables, int max_blocks_per_seq,
+                                   const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                   int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                                   float* partial_out, float* partial_lse, int max_partitions, int dtype,
+                                   void* stream) {
+    return decode_checked(true, out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+                          alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
+                          partial_lse, max_partitions, dtype, stream);
+}
+
+int opt_gqa_paged_attention_decode_simt(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                        const int32_t* block_tables, int max_blocks_per_seq,
+                                        const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                        int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                                        float* partial_out, float* partial_lse, int max_partitions, int dtype,
+                                        void* stream) {
+    return decode_checked(false, out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+                          alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
+                          partial_lse, max_partitions, dtype, stream);
 }
 
 int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const float* partial_lse,

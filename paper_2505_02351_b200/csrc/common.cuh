@@ -115,6 +115,13 @@ int launch_decode(void* out, const void* q, const void* k_cache, const void* v_c
                   int B, int Hq, int Hkv, int D, int bs, int partition_size, float* partial_out,
                   float* partial_lse, int max_partitions, int dtype, int* device_status, cudaStream_t stream);
 
+// bf16 only: the query group as rows of tensor-core tiles (decode_tc.cu).
+int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                     int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
+                     int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                     float* partial_out, float* partial_lse, int max_partitions, int* device_status,
+                     cudaStream_t stream);
+
 int launch_reduce(void* out, const float* partial_out, const float* partial_lse, const int32_t* context_lens,
                   int B, int Hq, int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream);
 

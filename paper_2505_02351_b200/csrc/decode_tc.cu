@@ -1,0 +1,412 @@
+// Paged GQA-ALiBi decode attention for bf16 caches on sm_100a, group-as-tile form
+// (Algorithm 2, "Compute context attention with caches"; Eq. 3-5; long-sequence
+// partitioning).
+//
+// Same decomposition as the SIMT kernel in decode.cu -- one CTA per (context
+// partition, KV head, sequence), every K/V tile brought on-chip once for the whole
+// query group, one private two-stage ring per warp -- but the G query heads of the
+// group are the rows of an m16n8k16 tile, so that Eq. 3's dot products and Eq. 5's
+// weighted sum run on the tensor pipe and the ALUs only see the softmax.  With G = 8
+// the arithmetic intensity is 8 flop per cache byte, which the fp32 FMA pipe cannot
+// sustain at HBM speed (measured: 40 % of the copy bandwidth at 46 % issue-slot use).
+//
+// Tiles are fetched by 2-D TMA with the 128-byte swizzle, which makes both the
+// row-wise ldmatrix of K (B operand of q k^T) and the transposing ldmatrix of V
+// (B operand of p V) bank-conflict free.  Scores stay in fp32 registers; p is
+// rounded to bf16 only as the tensor-core operand and the denominator sums the same
+// rounded values; accumulation is fp32.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace optgqa {
+
+namespace {
+
+constexpr int kTileTok = 16;
+constexpr int kWarps = 4;
+constexpr int kStages = 2;
+constexpr unsigned kFull = 0xffffffffu;
+
+struct TcParams {
+    void* out;
+    const __nv_bfloat16* q;
+    const int32_t* block_tables;
+    const int32_t* context_lens;
+    const float* slopes;
+    float* partial_out;
+    float* partial_lse;
+    int* status;
+    float scale;
+    int max_blocks;
+    int Hq;
+    int Hkv;
+    int bs;
+    int partition_size;
+    int max_partitions;
+};
+
+template <int D, int G>
+struct TcCfg {
+    static constexpr int NBOX = D / 64;                   // 128-byte-wide boxes per token row
+    static constexpr int BOX_BYTES = kTileTok * 128;      // 16 rows x 128 B
+    static constexpr int TILE_BYTES = NBOX * BOX_BYTES;   // K (or V) bytes per tile
+    static constexpr int WARP_RING = kStages * 2 * TILE_BYTES;
+    static constexpr int OFF_M = kWarps * WARP_RING;
+    static constexpr int OFF_L = OFF_M + kWarps * G * 4;
+    static constexpr int OFF_BAR = (OFF_L + kWarps * G * 4 + 7) & ~7;
+    static constexpr int SMEM = OFF_BAR + kWarps * kStages * 8 + 1024;   // + slack to align the ring to 1 KB
+    static_assert(G * D * 4 <= WARP_RING, "merge buffer must fit in the warp's ring");
+};
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+// d += a * b, m16n8k16, bf16 operands, fp32 accumulate.  Rows 8..15 of a are zero here (a1 = a3 = 0).
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+// Byte offset of 16-byte chunk `chunk` (0 .. D/8-1) of token row `row` inside a tile stored as
+// NBOX boxes of 16 rows x 128 B with the 128-byte swizzle (chunk index XOR row mod 8).
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+    return (uint32_t)((chunk >> 3) * (kTileTok * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(kWarps * 32, 3)
+decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                 const TcParams p) {
+    using C = TcCfg<D, G>;
+    constexpr int KS = D / 16;    // k-steps of q k^T
+    constexpr int NT = D / 8;     // n-tiles of p V
+    extern __shared__ char smem_raw[];
+    char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+
+    const int part = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;      // fragment row (query head of the group) and column pair
+    const int n = p.context_lens[s];
+    const bool split = p.partition_size > 0;
+    const int t0 = split ? part * p.partition_size : 0;
+    const int t1 = split ? min(t0 + p.partition_size, n) : n;
+
+    if (t0 >= t1) {
+        if (!split) {
+            __nv_bfloat16* o = static_cast<__nv_bfloat16*>(p.out) + ((size_t)s * p.Hq + (size_t)kvh * G) * D;
+            for (int e = threadIdx.x; e < G * D; e += blockDim.x) o[e] = __float2bfloat16_rn(0.f);
+        }
+        return;
+    }
+
+    char* ring = smem + warp * C::WARP_RING;
+    float* mbuf = reinterpret_cast<float*>(smem + C::OFF_M);
+    float* lbuf = reinterpret_cast<float*>(smem + C::OFF_L);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR) + warp * kStages;
+
+    const int tpp = p.bs / kTileTok;
+    const int first_tile = t0 / kTileTok;
+    const int ntiles = (t1 + kTileTok - 1) / kTileTok - first_tile;
+    const int cnt = ntiles > warp ? (ntiles - warp + kWarps - 1) / kWarps : 0;
+    const int32_t* table = p.block_tables + (size_t)s * p.max_blocks;
+
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < kStages; ++i) mbar_init(&bars[i], 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+
+    auto load_pages = [&](int kb) -> int {
+        int k = kb + lane;
+        return k < cnt ? __ldg(table + (first_tile + warp + k * kWarps) / tpp) : 0;
+    };
+    int pages_cur = load_pages(0), pages_next = load_pages(32), blk = 0;
+
+    auto issue = [&](int k) {
+        if ((k >> 5) != blk) {
+            pages_cur = pages_next;
+            ++blk;
+            pages_next = load_pages((blk + 1) * 32);
+        }
+        const int phys = __shfl_sync(kFull, pages_cur, k & 31);
+        if (lane == 0) {
+            const int tt = first_tile + warp + k * kWarps;
+            const int row = (phys * p.Hkv + kvh) * p.bs + (tt % tpp) * kTileTok;   // row of the [rows, D] view
+            char* dst = ring + (k % kStages) * 2 * C::TILE_BYTES;
+            uint64_t* bar = &bars[k % kStages];
+            mbar_expect_tx(bar, 2 * C::TILE_BYTES);
+#pragma unroll
+            for (int b = 0; b < C::NBOX; ++b) {
+                tma_load_2d(dst + b * C::BOX_BYTES, &map_k, b * 64, row, bar);
+                tma_load_2d(dst + C::TILE_BYTES + b * C::BOX_BYTES, &map_v, b * 64, row, bar);
+            }
+        }
+    };
+
+#pragma unroll
+    for (int k = 0; k < kStages; ++k)
+        if (k < cnt) issue(k);
+
+    // A fragments of q (rows = heads of the group; rows >= G are zero): a0 = dims 16s+2t,+1; a2 = dims 16s+8+2t,+1.
+    uint32_t qa[KS][2];
+    {
+        const uint32_t* qh =
+            reinterpret_cast<const uint32_t*>(p.q + ((size_t)s * p.Hq + (size_t)kvh * G + (g < G ? g : 0)) * D);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qa[ks][0] = g < G ? qh[ks * 8 + t] : 0u;
+            qa[ks][1] = g < G ? qh[ks * 8 + 4 + t] : 0u;
+        }
+    }
+    const float qscale = p.scale * kLog2e;
+    const float slope2 = (p.slopes && g < G) ? p.slopes[kvh * G + g] * kLog2e : 0.f;
+
+    float o[NT][4];
+#pragma unroll
+    for (int i = 0; i < NT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    int k = 0;
+
+    // ldmatrix lane roles: lane supplies the address of row (lane & 7) of matrix (lane >> 3).
+    const int lrow = lane & 7, lmat = lane >> 3;
+
+    for (; k < cnt; ++k) {
+        const int st = k % kStages;
+        char* kst = ring + st * 2 * C::TILE_BYTES;
+        char* vst = kst + C::TILE_BYTES;
+        ok = __all_sync(kFull, mbar_wait(&bars[st], (k / kStages) & 1, p.status));
+        if (!ok) break;
+
+        const int j0 = (first_tile + warp + k * kWarps) * kTileTok;
+        const int valid = min(kTileTok, t1 - j0);
+        if (valid < kTileTok) {
+            // zero the V rows past the end of the sequence (whole rows, so the swizzle does not matter)
+            for (int r = valid + (lane >> 3); r < kTileTok; r += 4)
+#pragma unroll
+                for (int b = 0; b < C::NBOX; ++b)
+                    *reinterpret_cast<uint4*>(vst + b * C::BOX_BYTES + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+            __syncwarp();
+        }
+
+        // ---- scores: S[head][token] for tokens j0 .. j0+15 as two n-tiles of 8
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+            const uint32_t kbase = smem_u32(kst);
+            const int krow = lrow + 8 * (lmat >> 1);          // matrices 0,1: tokens 0-7; 2,3: tokens 8-15
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t b[4];
+                ldmatrix_x4(b, kbase + swz(krow, 2 * ks + (lmat & 1)));
+                mma_bf16(sa, qa[ks][0], qa[ks][1], b[0], b[1]);
+                mma_bf16(sb, qa[ks][0], qa[ks][1], b[2], b[3]);
+            }
+        }
+        // thread holds head g, tokens j0 + {2t, 2t+1} (sa[0], sa[1]) and j0 + 8 + {2t, 2t+1} (sb[0], sb[1])
+        float sc[4];
+        {
+            const int ja = j0 + 2 * t, jb = ja + 8;
+            const float rel = (float)(ja - (n - 1));
+            sc[0] = fmaf(sa[0], qscale, slope2 * rel);
+            sc[1] = fmaf(sa[1], qscale, slope2 * (rel + 1.f));
+            sc[2] = fmaf(sb[0], qscale, slope2 * (rel + 8.f));
+            sc[3] = fmaf(sb[1], qscale, slope2 * (rel + 9.f));
+            sc[0] = ja < t1 ? sc[0] : -INFINITY;
+            sc[1] = ja + 1 < t1 ? sc[1] : -INFINITY;
+            sc[2] = jb < t1 ? sc[2] : -INFINITY;
+            sc[3] = jb + 1 < t1 ? sc[3] : -INFINITY;
+        }
+        float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
+        mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
+        const float m_new = fmaxf(m, mx);
+        const float alpha = ex2(m - m_new);
+        const bool rescale = __any_sync(kFull, m_new > m);
+        m = m_new;
+        // p rounded to bf16 once: the same values feed the tensor core and the denominator
+        const __nv_bfloat162 p01 = __floats2bfloat162_rn(ex2(sc[0] - m_new), ex2(sc[1] - m_new));
+        const __nv_bfloat162 p23 = __floats2bfloat162_rn(ex2(sc[2] - m_new), ex2(sc[3] - m_new));
+        const float2 f01 = __bfloat1622float2(p01), f23 = __bfloat1622float2(p23);
+        l = fmaf(l, alpha, (f01.x + f01.y) + (f23.x + f23.y));
+        const uint32_t pa0 = *reinterpret_cast<const uint32_t*>(&p01);
+        const uint32_t pa2 = *reinterpret_cast<const uint32_t*>(&p23);
+        if (rescale) {
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                o[i][0] *= alpha;
+                o[i][1] *= alpha;
+            }
+        }
+
+        // ---- O[head][dim] += P[head][token] * V[token][dim]; V transposed on the fly by ldmatrix.trans
+        {
+            const uint32_t vbase = smem_u32(vst);
+            const int vrow = lrow + 8 * (lmat & 1);           // matrices 0,2: tokens 0-7; 1,3: tokens 8-15
+#pragma unroll
+            for (int jj = 0; jj < NT / 2; ++jj) {
+                uint32_t b[4];
+                ldmatrix_x4_trans(b, vbase + swz(vrow, 2 * jj + (lmat >> 1)));
+                mma_bf16(o[2 * jj], pa0, pa2, b[0], b[1]);
+                mma_bf16(o[2 * jj + 1], pa0, pa2, b[2], b[3]);
+            }
+        }
+
+        __syncwarp();
+        if (k + kStages < cnt) {
+            fence_proxy_async();
+            issue(k + kStages);
+        }
+    }
+
+    if (!ok) {
+        for (int kk = k; kk < min(cnt, k + kStages); ++kk) mbar_wait(&bars[kk % kStages], (kk / kStages) & 1, p.status);
+    }
+
+    // ---- per-head denominator over the quad, then park (m, l, O) in this warp's ring for the CTA-wide merge
+    l += __shfl_xor_sync(kFull, l, 1);
+    l += __shfl_xor_sync(kFull, l, 2);
+    float* macc = reinterpret_cast<float*>(ring);
+    if (g < G) {
+#pragma unroll
+        for (int i = 0; i < NT; ++i) *reinterpret_cast<float2*>(macc + g * D + i * 8 + 2 * t) = make_float2(o[i][0], o[i][1]);
+        if (t == 0) {
+            mbuf[warp * G + g] = m;
+            lbuf[warp * G + g] = l;
+        }
+    }
+    __syncthreads();
+
+    const int nw = min(kWarps, ntiles);
+    for (int e = threadIdx.x; e < G * D; e += blockDim.x) {
+        const int hg = e / D, d = e % D;
+        float M = mbuf[hg];
+        for (int w = 1; w < nw; ++w) M = fmaxf(M, mbuf[w * G + hg]);
+        float num = 0.f, den = 0.f;
+        for (int w = 0; w < nw; ++w) {
+            const float f = ex2(mbuf[w * G + hg] - M);
+            den = fmaf(f, lbuf[w * G + hg], den);
+            num = fmaf(f, reinterpret_cast<const float*>(smem + w * C::WARP_RING)[e], num);
+        }
+        const float r = num / den;
+        const size_t row = (size_t)s * p.Hq + (size_t)kvh * G + hg;
+        if (split) {
+            p.partial_out[(row * p.max_partitions + part) * D + d] = r;
+            if (d == 0) p.partial_lse[row * p.max_partitions + part] = (M + log2f(den)) * kLn2;
+        } else {
+            static_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(r);
+        }
+    }
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// The cache seen as a 2-D bf16 tensor [num_blocks*Hkv*bs rows, D]; a box is 16 token rows x 64 dims (128 B).
+bool make_map(CUtensorMap* map, const void* cache, uint64_t rows, int D) {
+    EncodeFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTileTok};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, int G>
+int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, int B, cudaStream_t stream) {
+    using C = TcCfg<D, G>;
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    if (dev < 64 && !configured[dev]) {
+        if (cudaFuncSetAttribute(decode_tc_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
+            return OPT_GQA_ERR_CUDA;
+        configured[dev] = true;
+    }
+    dim3 grid(p.partition_size > 0 ? p.max_partitions : 1, p.Hkv, B);
+    decode_tc_kernel<D, G><<<grid, kWarps * 32, C::SMEM, stream>>>(mk, mv, p);
+    return cudaGetLastError() == cudaSuccess ? OPT_GQA_OK : OPT_GQA_ERR_CUDA;
+}
+
+template <int D>
+int launch_g(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, int B, int G, cudaStream_t stream) {
+    switch (G) {
+        case 1: return launch_one<D, 1>(mk, mv, p, B, stream);
+        case 2: return launch_one<D, 2>(mk, mv, p, B, stream);
+        case 4: return launch_one<D, 4>(mk, mv, p, B, stream);
+        case 8: return launch_one<D, 8>(mk, mv, p, B, stream);
+    }
+    return OPT_GQA_ERR_SHAPE;
+}
+
+}  // namespace
+
+int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                     int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
+                     int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                     float* partial_out, float* partial_lse, int max_partitions, int* device_status,
+                     cudaStream_t stream) {
+    const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
+    if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
+    CUtensorMap mk, mv;
+    if (!make_map(&mk, k_cache, rows, D) || !make_map(&mv, v_cache, rows, D)) return OPT_GQA_ERR_CUDA;
+    TcParams p;
+    p.out = out;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.block_tables = block_tables;
+    p.context_lens = context_lens;
+    p.slopes = alibi_slopes;
+    p.partial_out = partial_out;
+    p.partial_lse = partial_lse;
+    p.status = device_status;
+    p.scale = scale;
+    p.max_blocks = max_blocks_per_seq;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.bs = bs;
+    p.partition_size = partition_size;
+    p.max_partitions = max_partitions;
+    const int G = Hq / Hkv;
+    if (D == 128) return launch_g<128>(mk, mv, p, B, G, stream);
+    if (D == 64) return launch_g<64>(mk, mv, p, B, G, stream);
+    return OPT_GQA_ERR_SHAPE;
+}
+
+}  // namespace optgqa

@@ -33,12 +33,14 @@ def test_config1_poisoned_unused_slots():
 def test_config2_bf16_llama7b_like():
     _check(W.make_config(2))
     _check(W.make_config(2, poison=True), partition_size=256)
+    _check(W.make_config(2, poison=True), partition_size=256, simt=True)
 
 
 def test_config3_long_sequence_partitioned():
     wl = W.make_config(3)
     assert wl.partition_size == 512
     _check(wl)
+    _check(wl, simt=True)
 
 
 def test_config4_ragged_large_batch_with_append():
@@ -57,12 +59,16 @@ def test_shape_matrix(dtype, D, Hq, Hkv, bs):
     _check(wl)
     _check(wl, partition_size=64)
     _check(wl, partition_size=0, slopes=False)
+    if dtype == "bf16":        # the CUDA-core kernel on bf16 caches (fp32 always runs on it)
+        _check(wl, simt=True)
+        _check(wl, partition_size=64, simt=True)
 
 
 @pytest.mark.parametrize("P", [16, 48, 512, 4096])
 def test_any_partition_size_agrees_with_single_pass(P):
     wl = W.make_custom("p", "bf16", 8, 2, 128, 16, [700, 33, 2049], seed=21)
     _check(wl, partition_size=P)
+    _check(wl, partition_size=P, simt=True)
 
 
 def test_partials_match_the_oracle_partials():

@@ -22,23 +22,24 @@ class DeviceWorkload:
         self.out = torch.full_like(self.q, float("nan"))
 
 
-def gpu_decode(wl: W.Workload, partition_size=None, append=True, slopes=True):
+def gpu_decode(wl: W.Workload, partition_size=None, append=True, slopes=True, simt=False):
     """append + decode (+ reduce) through the C ABI; returns (out float64 numpy, DeviceWorkload)."""
     d = DeviceWorkload(wl)
     P = wl.partition_size if partition_size is None else partition_size
     if append:
         binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
     sl = d.alibi_slopes if slopes else None
+    decode = binding.paged_attention_decode_simt if simt else binding.paged_attention_decode
     if P > 0:
         maxP = max(1, (int(wl.context_lens.max()) + P - 1) // P) if wl.B else 1
         po = torch.full((wl.B, wl.Hq, maxP, wl.D), float("nan"), device="cuda:0", dtype=torch.float32)
         pl = torch.full((wl.B, wl.Hq, maxP), float("nan"), device="cuda:0", dtype=torch.float32)
-        binding.paged_attention_decode(None, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, sl, wl.scale,
+        decode(None, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, sl, wl.scale,
                                        partition_size=P, partial_out=po, partial_lse=pl, max_partitions=maxP)
         binding.paged_attention_reduce(d.out, po, pl, d.context_lens, P)
         d.partial_out, d.partial_lse = po, pl
     else:
-        binding.paged_attention_decode(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, sl, wl.scale)
+        decode(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, sl, wl.scale)
     torch.cuda.synchronize()
     assert binding.device_status() == 0
     return d.out.double().cpu().numpy(), d
@@ -55,7 +56,7 @@ def oracle_inputs(wl: W.Workload, append=True):
                 qsl=None if wl.q_start_loc is None else wl.q_start_loc.numpy())
 
 
-def oracle_attention(wl: W.Workload, append=True, slopes=True):
+def oracle_attention(wl: W.Workload, append=True, slopes=True, simt=False):
     a = oracle_inputs(wl, append)
     return oracle.paged_attention(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"] if slopes else None, wl.scale,
                                   wl.dtype, q_start_loc=a["qsl"])
