@@ -212,9 +212,16 @@ def check(rc: int, what: str):
         raise RuntimeError(f"{what} failed with status {rc}")
 
 
+EVENT_EVERY = 8   # every 8th timed step brackets its decode launch with CUDA events
+
+
 def run_timed(batch: DeviceBatch, steps: int, warmup: int, per_kernel_events: bool):
     """Warm-up, then `steps` steps timed with CUDA events on the launching stream.
 
+    A step is one opt_gqa_decode_step call (append -> decode -> reduce, chained with programmatic
+    dependent launches).  Every EVENT_EVERY-th step is issued as the three separate calls instead, with
+    an event before and after the decode launch: those samples give the decode kernel's average
+    duration inside the timed region without putting event records between the kernels of every step.
     Returns (total_ms, decode_ms_avg or None, launches).  Consecutive steps use different pool copies.
     """
     import torch
@@ -224,35 +231,38 @@ def run_timed(batch: DeviceBatch, steps: int, warmup: int, per_kernel_events: bo
     lib, R, split = batch.lib, len(batch.k_pools), batch.P > 0
     a_app = [batch.args_append(i, sh) for i in range(R)]
     a_dec = [batch.args_decode(i, sh) for i in range(R)]
+    a_step = [batch.args_step(i, sh) for i in range(R)]
     a_red = batch.args_reduce(sh) if split else None
     f_app, f_dec, f_red = lib.opt_gqa_cache_append, lib.opt_gqa_paged_attention_decode, lib.opt_gqa_paged_attention_reduce
+    f_step = lib.opt_gqa_decode_step
 
     def step(i, ev=None):
+        if ev is None:
+            check(f_step(*a_step[i % R]), "decode_step")
+            return
         check(f_app(*a_app[i % R]), "cache_append")
-        if ev is not None:
-            ev[0].record(stream)
+        ev[0].record(stream)
         check(f_dec(*a_dec[i % R]), "decode")
-        if ev is not None:
-            ev[1].record(stream)
+        ev[1].record(stream)
         if split:
             check(f_red(*a_red), "reduce")
 
     for i in range(warmup):
         step(i)
     torch.cuda.synchronize()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)] \
-        if per_kernel_events else None
+    evs = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for i in range(0, steps, EVENT_EVERY)} if per_kernel_events else {}
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     torch.cuda.synchronize()
     start.record(stream)
     for i in range(steps):
-        step(warmup + i, evs[i] if evs else None)
+        step(warmup + i, evs.get(i))
     end.record(stream)
     torch.cuda.synchronize()
     barrier()
     total_ms = start.elapsed_time(end)
-    dec_ms = sum(a.elapsed_time(b) for a, b in evs) / steps if evs else None
+    dec_ms = sum(a.elapsed_time(b) for a, b in evs.values()) / len(evs) if evs else None
     return total_ms, dec_ms, steps * (3 if split else 2)
 
 

@@ -11,6 +11,7 @@ __global__ void __launch_bounds__(256)
 cache_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* __restrict__ k_cache,
                     uint4* __restrict__ v_cache, const int64_t* __restrict__ slot_mapping, long long total_vecs,
                     int Hkv, int row_vecs, int bs) {
+    grid_dependency_launch();   // the attention grid may start its prologue; it waits before reading the cache
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total_vecs) return;
     int vec = (int)(i % row_vecs);

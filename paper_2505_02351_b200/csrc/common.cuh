@@ -83,6 +83,25 @@ __device__ __forceinline__ float lg2(float x) {
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Launch that may begin while the preceding kernel of the stream is still draining (programmatic
+// stream serialisation).  The kernel must execute grid_dependency_wait() before it touches anything
+// the preceding kernel writes; with a predecessor that never signals, this is an ordinary launch.
+template <typename... KArgs, typename... Args>
+inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                            Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) == cudaSuccess ? OPT_GQA_OK : OPT_GQA_ERR_CUDA;
+}
+
 // ----------------------------------------------------------------------------- storage types
 // Two adjacent bf16 values packed in one 32-bit word -> (low element, high element) as fp32.
 __device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {

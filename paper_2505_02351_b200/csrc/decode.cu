@@ -135,9 +135,9 @@ __global__ void __launch_bounds__(kWarps * 32, DecodeCfg<T, D, G>::MIN_CTAS)
 decode_kernel(const DecodeParams p) {
     using C = DecodeCfg<T, D, G>;
     constexpr int NC2 = C::NC2;
-    constexpr int EPL = C::EPL;
     extern __shared__ __align__(128) char smem[];
 
+    grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
     const int part = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, c = lane & 15;
@@ -201,6 +201,7 @@ decode_kernel(const DecodeParams p) {
         }
     };
 
+    grid_dependency_wait();     // the cache may still be receiving this step's appended tokens
 #pragma unroll
     for (int k = 0; k < kStages; ++k)
         if (k < cnt) issue(k);
@@ -382,8 +383,7 @@ static int launch_one(const DecodeParams& p, int B, cudaStream_t stream) {
         configured[dev] = true;
     }
     dim3 grid(p.partition_size > 0 ? p.max_partitions : 1, p.Hkv, B);
-    decode_kernel<T, D, G><<<grid, kWarps * 32, C::SMEM, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? OPT_GQA_OK : OPT_GQA_ERR_CUDA;
+    return launch_dependent(decode_kernel<T, D, G>, grid, dim3(kWarps * 32), C::SMEM, stream, p);
 }
 
 template <typename T, int D>

@@ -23,9 +23,9 @@ namespace optgqa {
 
 namespace {
 
-constexpr int kTileTok = 16;
-constexpr int kWarps = 4;
-constexpr int kStages = 2;
+constexpr int kTileTok = 16;   // tokens per tile (one ring stage holds a K tile and a V tile)
+constexpr int kWarps = 4;      // warps per CTA, each with a private ring
+constexpr int kStages = 2;     // ring depth per warp
 constexpr unsigned kFull = 0xffffffffu;
 
 struct TcParams {
@@ -103,6 +103,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     extern __shared__ char smem_raw[];
     char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
 
+    grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
     const int part = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;      // fragment row (query head of the group) and column pair
@@ -164,6 +165,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         }
     };
 
+    grid_dependency_wait();     // the cache may still be receiving this step's appended tokens
 #pragma unroll
     for (int k = 0; k < kStages; ++k)
         if (k < cnt) issue(k);
@@ -361,8 +363,7 @@ int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, 
         configured[dev] = true;
     }
     dim3 grid(p.partition_size > 0 ? p.max_partitions : 1, p.Hkv, B);
-    decode_tc_kernel<D, G><<<grid, kWarps * 32, C::SMEM, stream>>>(mk, mv, p);
-    return cudaGetLastError() == cudaSuccess ? OPT_GQA_OK : OPT_GQA_ERR_CUDA;
+    return launch_dependent(decode_tc_kernel<D, G>, grid, dim3(kWarps * 32), C::SMEM, stream, mk, mv, p);
 }
 
 template <int D>
