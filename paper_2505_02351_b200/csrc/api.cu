@@ -126,15 +126,16 @@ int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_s
                                     int64_t num_blocks, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
-    if (B < 0 || max_q_len < 0 || !shape_ok(Hq, Hkv, D, bs) || D != 128 || max_blocks_per_seq < 0 || num_blocks < 0)
+    if (B < 0 || max_q_len < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0)
         return OPT_GQA_ERR_SHAPE;
     if (B == 0 || max_q_len == 0) return OPT_GQA_OK;
+    if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
     if (!out || !q || !q_start_loc || !k_cache || !v_cache || !block_tables || !context_lens) return OPT_GQA_ERR_NULL;
     if (!aligned16(out) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
     return launch_prefill(out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables, max_blocks_per_seq,
-                          context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, status,
+                          context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, status,
                           static_cast<cudaStream_t>(stream));
 }
 

@@ -147,6 +147,6 @@ int launch_reduce(void* out, const float* partial_out, const float* partial_lse,
 int launch_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len, const void* k_cache,
                    const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
                    const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
-                   int D, int bs, int* device_status, cudaStream_t stream);
+                   int D, int bs, int64_t num_blocks, int* device_status, cudaStream_t stream);
 
 }  // namespace optgqa

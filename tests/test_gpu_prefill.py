@@ -1,0 +1,69 @@
+"""Parity of the tensor-core chunked-prefill variant (append -> prefill, through the C ABI) with the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_02351_b200 import binding
+from paper_2505_02351_b200 import workloads as W
+from tests import util
+
+pytestmark = pytest.mark.gpu
+TOL = util.TOL["bf16"]
+
+
+def _check(wl, **kw):
+    got, d = util.gpu_prefill(wl, **kw)
+    want = util.oracle_attention(wl, **kw)
+    assert np.isfinite(got).all()
+    err = np.max(np.abs(got - want)) if got.size else 0.0
+    assert err <= TOL, f"{wl.name}: max-abs error {err}"
+    return got, want, d
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (4, 2), (8, 2), (8, 1)])
+@pytest.mark.parametrize("bs", [16, 32])
+def test_shape_matrix_ragged_chunks(D, Hq, Hkv, bs):
+    # new-token counts that end inside a query block, span several, equal the context (no history), or are 1
+    lens = [200, 77, 33, 130, 1, 64, 300]
+    qls = [70, 77, 1, 129, 1, 16, 17]
+    wl = W.make_custom("pf", "bf16", Hq, Hkv, D, bs, lens, q_lens=qls, seed=D + Hq + bs, poison=True)
+    _check(wl)
+    _check(wl, slopes=False)
+
+
+def test_config5_shrunk():
+    # the named workload with every length divided by 8: 512 existing + 256 new tokens per sequence
+    wl = W.make_config(5, shrink=8, poison=True)
+    assert wl.T == 4 * 256
+    _check(wl)
+
+
+def test_prefill_with_one_new_token_is_the_decode_result():
+    wl = W.make_custom("pf1", "bf16", 8, 2, 128, 16, [300, 41, 1000], q_lens=[1, 1, 1], seed=31)
+    got, _ = util.gpu_prefill(wl)
+    wl_dec = W.Workload(**{**wl.__dict__, "q_start_loc": None})
+    dec, _ = util.gpu_decode(wl_dec)
+    want = util.oracle_attention(wl)
+    assert np.max(np.abs(got - want)) <= TOL
+    assert np.max(np.abs(got - dec)) <= TOL
+
+
+def test_empty_sequences_and_no_new_tokens():
+    # a sequence that contributes no new tokens leaves no row; the others are unaffected
+    wl = W.make_custom("pf0", "bf16", 4, 2, 128, 16, [50, 64, 20], q_lens=[0, 64, 20], seed=32, poison=True)
+    _check(wl)
+
+
+def test_config5_full_size_sampled_rows():
+    """The full workload in the configuration the benchmark times; the oracle checks sampled rows one by one."""
+    wl = W.make_config(5)
+    got, _ = util.gpu_prefill(wl)
+    assert np.isfinite(got).all()
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([rng.integers(0, wl.T, size=24), [0, 2047, 2048, wl.T - 1]]))
+    want = util.oracle_prefill_rows(wl, rows)
+    err = np.max(np.abs(got[rows] - want))
+    assert err <= TOL, err
+    # property that holds at any size: every output lies in the convex hull of V's value range
+    assert np.abs(got).max() <= float(wl.v_cache.float().abs().max().item()) + float(wl.v_new.float().abs().max().item())

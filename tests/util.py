@@ -60,3 +60,30 @@ def oracle_attention(wl: W.Workload, append=True, slopes=True, simt=False):
     a = oracle_inputs(wl, append)
     return oracle.paged_attention(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"] if slopes else None, wl.scale,
                                   wl.dtype, q_start_loc=a["qsl"])
+
+
+def gpu_prefill(wl: W.Workload, append=True, slopes=True):
+    """append + chunked prefill through the C ABI; returns (out float64 numpy, DeviceWorkload)."""
+    d = DeviceWorkload(wl)
+    if append:
+        binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
+    qsl = wl.q_start_loc.numpy()
+    max_q_len = int((qsl[1:] - qsl[:-1]).max()) if wl.B else 0
+    binding.paged_attention_prefill(d.out, d.q, d.q_start_loc, max_q_len, d.k_cache, d.v_cache, d.block_tables,
+                                    d.context_lens, d.alibi_slopes if slopes else None, wl.scale)
+    torch.cuda.synchronize()
+    assert binding.device_status() == 0
+    return d.out.double().cpu().numpy(), d
+
+
+def oracle_prefill_rows(wl: W.Workload, rows, append=True, slopes=True):
+    """Oracle output for selected new-token rows only: row t of sequence s is a decode query at
+    position pos_t over the context truncated to pos_t + 1 tokens (the oracle's decode mode)."""
+    a = oracle_inputs(wl, append)
+    qsl = a["qsl"]
+    seq = np.searchsorted(qsl, rows, side="right") - 1
+    qlen = qsl[seq + 1] - qsl[seq]
+    pos = a["n"][seq] - qlen + (np.asarray(rows) - qsl[seq])
+    return oracle.paged_attention(np.ascontiguousarray(a["q"][rows]), a["k"], a["v"],
+                                  np.ascontiguousarray(a["bt"][seq]), (pos + 1).astype(np.int32),
+                                  a["slopes"] if slopes else None, wl.scale, wl.dtype)
