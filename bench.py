@@ -166,8 +166,9 @@ class DeviceBatch:
         self.maxP = max(1, (int(wl.context_lens.max()) + partition_size - 1) // partition_size) if partition_size else 1
         ws = binding.workspace_bytes(wl.B, wl.Hq, wl.D, self.maxP) if partition_size else 0
         self.workspace = torch.empty(max(ws, 16), dtype=torch.uint8, device=device)
-        self.partial_out = self.workspace[: wl.B * wl.Hq * self.maxP * wl.D * 4].view(torch.float32)
-        self.partial_lse = self.workspace[wl.B * wl.Hq * self.maxP * wl.D * 4: ws].view(torch.float32) if ws else None
+        npart = wl.B * wl.Hq * self.maxP
+        self.partial_out = self.workspace[: npart * wl.D * 4].view(torch.float32)
+        self.partial_lse = self.workspace[npart * wl.D * 4: npart * (wl.D + 1) * 4].view(torch.float32) if ws else None
         self.lib = binding.load()
         self.dt = binding.BF16 if wl.dtype == "bf16" else binding.FP32
 
@@ -177,8 +178,17 @@ class DeviceBatch:
         return (self.k_new.data_ptr(), self.v_new.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(),
                 self.slots.data_ptr(), wl.B, wl.Hkv, wl.D, wl.bs, wl.num_blocks, self.dt, stream)
 
+    @property
+    def balanced(self) -> bool:
+        """bf16 partitioned steps take the load-balanced split (what opt_gqa_decode_step runs)."""
+        return self.P > 0 and self.wl.dtype == "bf16"
+
     def args_decode(self, i, stream):
         wl = self.wl
+        if self.balanced:
+            return (self.q.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(), self.tables.data_ptr(),
+                    wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D,
+                    wl.bs, wl.num_blocks, self.P, self.workspace.data_ptr(), self.maxP, self.dt, stream)
         return (self.out.data_ptr(), self.q.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(),
                 self.tables.data_ptr(), wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B,
                 wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, self.P,
@@ -187,6 +197,9 @@ class DeviceBatch:
 
     def args_reduce(self, stream):
         wl = self.wl
+        if self.balanced:
+            return (self.out.data_ptr(), self.workspace.data_ptr(), self.lens.data_ptr(), wl.B, wl.Hq, wl.Hkv, wl.D,
+                    self.P, self.maxP, self.dt, stream)
         return (self.out.data_ptr(), self.partial_out.data_ptr(), self.partial_lse.data_ptr(), self.lens.data_ptr(),
                 wl.B, wl.Hq, wl.D, self.P, self.maxP, self.dt, stream)
 
@@ -205,6 +218,89 @@ class DeviceBatch:
         n = wl.context_lens.long()
         tables = int(((n + wl.bs - 1) // wl.bs).sum()) * 4
         return wl.kv_bytes() + 2 * wl.B * wl.Hq * wl.D * es + tables
+
+
+class PrefillBatch:
+    """The chunked-prefill workload resident in HBM: a step appends every sequence's new tokens, then attends."""
+
+    def __init__(self, wl, device):
+        import torch
+
+        from paper_2505_02351_b200 import binding
+
+        self.wl, self.dev = wl, device
+        to = lambda t: t.to(device)
+        self.q, self.k_new, self.v_new = to(wl.q), to(wl.k_new), to(wl.v_new)
+        self.slots, self.tables, self.lens = to(wl.slot_mapping), to(wl.block_tables), to(wl.context_lens)
+        self.slopes, self.qsl = to(wl.alibi_slopes), to(wl.q_start_loc)
+        self.k_pool, self.v_pool = to(wl.k_cache), to(wl.v_cache)
+        self.out = torch.zeros_like(self.q)
+        qsl = wl.q_start_loc.numpy()
+        self.max_q_len = int((qsl[1:] - qsl[:-1]).max())
+        self.lib = binding.load()
+
+    def flops(self) -> float:
+        """4*D flop (q.k and p.v) per unmasked (new token, key) pair per query head."""
+        wl = self.wl
+        qsl = wl.q_start_loc.numpy().astype("int64")
+        n = wl.context_lens.numpy().astype("int64")
+        pairs = 0
+        for s in range(wl.B):
+            ql = int(qsl[s + 1] - qsl[s])
+            first = int(n[s]) - ql + 1                       # keys seen by the first new token
+            pairs += ql * first + ql * (ql - 1) // 2
+        return 4.0 * wl.D * wl.Hq * pairs
+
+    def run(self, steps: int, warmup: int):
+        """Returns (ms per step, ms per prefill launch)."""
+        import torch
+
+        wl = self.wl
+        stream = torch.cuda.current_stream()
+        sh = stream.cuda_stream
+        a_app = (self.k_new.data_ptr(), self.v_new.data_ptr(), self.k_pool.data_ptr(), self.v_pool.data_ptr(),
+                 self.slots.data_ptr(), wl.T, wl.Hkv, wl.D, wl.bs, wl.num_blocks, 1, sh)
+        a_pf = (self.out.data_ptr(), self.q.data_ptr(), self.qsl.data_ptr(), self.max_q_len, self.k_pool.data_ptr(),
+                self.v_pool.data_ptr(), self.tables.data_ptr(), wl.max_blocks, self.lens.data_ptr(),
+                self.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, 1, sh)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(warmup + steps):
+            if i == warmup:
+                torch.cuda.synchronize()
+                start.record(stream)
+            check(self.lib.opt_gqa_cache_append(*a_app), "cache_append")
+            if i >= warmup:
+                evs[i - warmup][0].record(stream)
+            check(self.lib.opt_gqa_paged_attention_prefill(*a_pf), "prefill")
+            if i >= warmup:
+                evs[i - warmup][1].record(stream)
+        end.record(stream)
+        torch.cuda.synchronize()
+        return start.elapsed_time(end) / steps, sum(a.elapsed_time(b) for a, b in evs) / steps
+
+
+def measured_tensor_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+    except Exception:
+        return 1400.0, "fallback (sustained)"
+
+
+def prefill_report(dev, steps: int, warmup: int) -> dict:
+    """Side measurement of the chunked-prefill workload: append of the new tokens + tensor-core prefill."""
+    from paper_2505_02351_b200 import workloads as W
+
+    wl = W.make_config(5)
+    pb = PrefillBatch(wl, dev)
+    step_ms, pf_ms = pb.run(steps, warmup)
+    peak, kind = measured_tensor_peak()
+    tf = pb.flops() / (pf_ms * 1e-3) / 1e12
+    return {"new_tokens_per_s": wl.T / (step_ms * 1e-3), "ms_per_step": step_ms, "prefill_us": pf_ms * 1e3,
+            "prefill_TFLOPs": tf, "frac_of_bf16_peak": tf / peak, "peak": peak, "peak_kind": f"of {kind}",
+            "flop_per_launch": pb.flops(), "bound": "tensor"}
 
 
 def check(rc: int, what: str):
@@ -233,7 +329,11 @@ def run_timed(batch: DeviceBatch, steps: int, warmup: int, per_kernel_events: bo
     a_dec = [batch.args_decode(i, sh) for i in range(R)]
     a_step = [batch.args_step(i, sh) for i in range(R)]
     a_red = batch.args_reduce(sh) if split else None
-    f_app, f_dec, f_red = lib.opt_gqa_cache_append, lib.opt_gqa_paged_attention_decode, lib.opt_gqa_paged_attention_reduce
+    f_app = lib.opt_gqa_cache_append
+    if batch.balanced:
+        f_dec, f_red = lib.opt_gqa_paged_attention_decode_balanced, lib.opt_gqa_paged_attention_reduce_balanced
+    else:
+        f_dec, f_red = lib.opt_gqa_paged_attention_decode, lib.opt_gqa_paged_attention_reduce
     f_step = lib.opt_gqa_decode_step
 
     def step(i, ev=None):
@@ -398,6 +498,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--no-extra", action="store_true", help="skip the short side measurements of the other workloads")
+    ap.add_argument("--prefill-only", action="store_true",
+                    help="run only the chunked-prefill side measurement and print its report (profiling runs)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
 
@@ -423,6 +525,10 @@ def main():
         import torch.distributed as dist
 
         dist.init_process_group("nccl", device_id=dev)
+    if args.prefill_only:
+        if rank == 0:
+            print(json.dumps(prefill_report(dev, args.steps or 20, max(3, args.warmup or 3))), flush=True)
+        return
     steps = args.steps if args.steps is not None else 4000
     warmup = max(3, args.warmup if args.warmup is not None else 50)
 
@@ -453,7 +559,7 @@ def main():
     peak, peak_kind = measured_peak()
     alg = batch.algorithmic_bytes()
     achieved = alg / (dec_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (balanced split)" if batch.balanced else "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(args.config),
                 "algorithmic_bytes_per_launch": alg, "kernel_us": dec_ms * 1e3,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
@@ -490,6 +596,7 @@ def main():
                               "frac_of_peak": a2 / (d_ms * 1e-3) / 1e9 / peak, "partition_size": b2.P}
             del b2, w2
             torch.cuda.empty_cache()
+        extra[W.CONFIG_NAMES[5]] = prefill_report(dev, 20, 3)
         line["other_workloads"] = extra
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

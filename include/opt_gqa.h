@@ -88,7 +88,7 @@ int opt_gqa_cache_append(const void* k_new, const void* v_new, void* k_cache, vo
  *   alibi_slopes  [Hq] fp32, or NULL for no bias
  *   partition_size  0: one CTA walks the whole sequence and writes out.
  *                   P > 0 (a multiple of 16): the long-sequence split described
- *                   before Eq. 1 -- CTA (s, kv head, p) attends to keys
+ *                   before Eq. 1 -- work item (s, kv head, p) attends to keys
  *                   [pP, min((p+1)P, n_s)) and writes, for each head of the group,
  *                   the normalised partial result and its log-sum-exp:
  *                     partial_out [B, Hq, max_partitions, D] fp32
@@ -118,6 +118,39 @@ int opt_gqa_paged_attention_decode_simt(void* out, const void* q, const void* k_
                                         int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
                                         int partition_size, float* partial_out, float* partial_lse,
                                         int max_partitions, int dtype, void* stream);
+
+/*
+ * Partitioned decode with a load-balanced split, bf16 caches only: the same result as
+ * opt_gqa_paged_attention_decode with partition_size = P followed by the reduce, but the
+ * context partitions (the split described before Eq. 1) are additionally cut wherever the
+ * share of one worker of the persistent grid ends, so that every SM streams the same number
+ * of cache bytes whatever the mix of sequence lengths.  Every piece lies inside one
+ * P-token partition of one (sequence, KV head); its normalised result and log-sum-exp go
+ * to `workspace` in a layout private to the library, and
+ * opt_gqa_paged_attention_reduce_balanced (same B, Hq, Hkv, D, partition_size,
+ * max_partitions, same workspace, later on the same stream) merges them into out.
+ *
+ *   workspace     opt_gqa_workspace_bytes(B, Hq, D, max_partitions) bytes, 16-byte aligned;
+ *                 contents need no initialisation and are overwritten
+ *   partition_size  P > 0, a multiple of 16;  max_partitions >= ceil(max_s n_s / P)
+ * Other arguments as in opt_gqa_paged_attention_decode.  dtype must be OPT_GQA_BF16.
+ */
+int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, const void* v_cache,
+                                            const int32_t* block_tables, int max_blocks_per_seq,
+                                            const int32_t* context_lens, const float* alibi_slopes, float scale,
+                                            int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                                            int partition_size, void* workspace, int max_partitions, int dtype,
+                                            void* stream);
+
+/*
+ * Log-sum-exp merge of the pieces written by opt_gqa_paged_attention_decode_balanced (the
+ * combination step of the paragraph before Eq. 1, over pieces instead of whole partitions):
+ *     out = sum_c e^{lse_c} o_c / sum_c e^{lse_c}   over the pieces c of the row's sequence and KV head.
+ * out [B, Hq, D] in `dtype`; n_s == 0 gives zero rows.
+ */
+int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B,
+                                            int Hq, int Hkv, int D, int partition_size, int max_partitions,
+                                            int dtype, void* stream);
 
 /*
  * Merge of the partitions' results (the paragraph before Eq. 1: each partition's
@@ -155,9 +188,10 @@ int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_s
  * B new tokens (k_new, v_new [B, Hkv, D], slot_mapping [B]), then decode, then --
  * when partition_size > 0 -- the reduce, all enqueued on `stream` by one call.
  * workspace: opt_gqa_workspace_bytes(B, Hq, D, max_partitions) bytes of device
- * memory (partial_out followed by partial_lse); may be NULL when partition_size
- * is 0.  Other arguments as in the three calls it chains.  out [B, Hq, D] is
- * always written.
+ * memory, 16-byte aligned; may be NULL when partition_size is 0.  bf16 caches take
+ * the balanced split (decode_balanced + reduce_balanced), fp32 caches one partial
+ * per partition (partial_out followed by partial_lse at the start of workspace).
+ * Other arguments as in the calls it chains.  out [B, Hq, D] is always written.
  */
 int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,
                         const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,
@@ -188,9 +222,11 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
 size_t opt_gqa_step_staging_bytes(int B, int Hq, int Hkv, int D, int max_blocks_per_seq, int dtype);
 
 /*
- * Bytes of fp32 scratch a split decode needs: partial_out followed by partial_lse,
- * B*Hq*max_partitions*(D+1) floats.  (Workspace sizing for the partitioning step;
- * pure host arithmetic.)  Returns 0 for non-positive arguments.
+ * Bytes of device scratch a split decode needs, whichever layout is used: one
+ * (D+1)-float row per (sequence, head, partition) -- partial_out followed by
+ * partial_lse -- or the balanced split's piece rows and bookkeeping, which add a
+ * fixed 16384 rows and less than 1 KB + 16*B bytes.  (Workspace sizing for the
+ * partitioning step; pure host arithmetic.)  Returns 0 for non-positive arguments.
  */
 size_t opt_gqa_workspace_bytes(int B, int Hq, int D, int max_partitions);
 

@@ -29,6 +29,9 @@ SIGNATURES = {
                                             _i, _vp, _vp, _i, _i, _vp]),
     "opt_gqa_paged_attention_decode_simt": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                                  _i, _vp, _vp, _i, _i, _vp]),
+    "opt_gqa_paged_attention_decode_balanced": (_i, [_vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
+                                                     _i, _vp, _i, _i, _vp]),
+    "opt_gqa_paged_attention_reduce_balanced": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_reduce": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_prefill": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i,
                                              _i, _i64, _i, _vp]),
@@ -131,6 +134,27 @@ def paged_attention_decode_simt(out, q, k_cache, v_cache, block_tables, context_
                                 max_partitions: int = 0, stream=None) -> None:
     _decode("opt_gqa_paged_attention_decode_simt", out, q, k_cache, v_cache, block_tables, context_lens,
             alibi_slopes, scale, partition_size, partial_out, partial_lse, max_partitions, stream)
+
+
+def paged_attention_decode_balanced(q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
+                                    partition_size: int, workspace, max_partitions: int, stream=None) -> None:
+    B, Hq, D = q.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    assert block_tables.dtype == torch.int32 and context_lens.dtype == torch.int32
+    assert alibi_slopes is None or alibi_slopes.dtype == torch.float32
+    assert workspace.numel() * workspace.element_size() >= workspace_bytes(B, Hq, D, max_partitions)
+    _check(load().opt_gqa_paged_attention_decode_balanced(
+        _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables), block_tables.shape[1], _ptr(context_lens),
+        _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, _ptr(workspace), max_partitions,
+        _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_decode_balanced")
+
+
+def paged_attention_reduce_balanced(out, workspace, context_lens, Hkv: int, partition_size: int, max_partitions: int,
+                                    stream=None) -> None:
+    B, Hq, D = out.shape
+    _check(load().opt_gqa_paged_attention_reduce_balanced(
+        _ptr(out), _ptr(workspace), _ptr(context_lens), B, Hq, Hkv, D, partition_size, max_partitions,
+        _DTYPE_CODE[out.dtype], _stream(stream)), "opt_gqa_paged_attention_reduce_balanced")
 
 
 def paged_attention_reduce(out, partial_out, partial_lse, context_lens, partition_size: int, stream=None) -> None:

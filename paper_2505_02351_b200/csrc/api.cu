@@ -74,6 +74,10 @@ static int decode_checked(bool allow_tensor_cores, void* out, const void* q, con
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (allow_tensor_cores && dtype == OPT_GQA_BF16 && partition_size > 0)
+        return launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
+                                    scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out, partial_lse,
+                                    nullptr, max_partitions, status, cs);
     if (allow_tensor_cores && dtype == OPT_GQA_BF16)
         return launch_decode_tc(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                                 alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
@@ -119,6 +123,43 @@ int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const fl
                          dtype, static_cast<cudaStream_t>(stream));
 }
 
+int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, const void* v_cache,
+                                            const int32_t* block_tables, int max_blocks_per_seq,
+                                            const int32_t* context_lens, const float* alibi_slopes, float scale,
+                                            int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                                            int partition_size, void* workspace, int max_partitions, int dtype,
+                                            void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0 || partition_size <= 0 ||
+        partition_size % 16 != 0 || max_partitions <= 0)
+        return OPT_GQA_ERR_SHAPE;
+    if (B > 65535 || Hkv > 65535 || max_partitions > 65535) return OPT_GQA_ERR_SHAPE;
+    if (B == 0) return OPT_GQA_OK;
+    if (!q || !k_cache || !v_cache || !block_tables || !context_lens || !workspace) return OPT_GQA_ERR_NULL;
+    if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(workspace)) return OPT_GQA_ERR_ALIGN;
+    int* status = device_status_ptr();
+    if (!status) return OPT_GQA_ERR_CUDA;
+    return launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
+                                scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, nullptr, nullptr, workspace,
+                                max_partitions, status, static_cast<cudaStream_t>(stream));
+}
+
+int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B,
+                                            int Hq, int Hkv, int D, int partition_size, int max_partitions,
+                                            int dtype, void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128) || partition_size <= 0 ||
+        partition_size % 16 != 0 || max_partitions <= 0)
+        return OPT_GQA_ERR_SHAPE;
+    if (B == 0) return OPT_GQA_OK;
+    if (!out || !workspace || !context_lens) return OPT_GQA_ERR_NULL;
+    if (!aligned16(out) || !aligned16(workspace)) return OPT_GQA_ERR_ALIGN;
+    return launch_reduce_balanced(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, dtype,
+                                  static_cast<cudaStream_t>(stream));
+}
+
 int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len,
                                     const void* k_cache, const void* v_cache, const int32_t* block_tables,
                                     int max_blocks_per_seq, const int32_t* context_lens,
@@ -149,6 +190,14 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
     int rc = opt_gqa_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, B, Hkv, D, bs, num_blocks, dtype,
                                   stream);
     if (rc != OPT_GQA_OK) return rc;
+    if (dtype == OPT_GQA_BF16 && partition_size > 0 && B > 0) {
+        rc = opt_gqa_paged_attention_decode_balanced(q, k_cache, v_cache, block_tables, max_blocks_per_seq,
+                                                     context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks,
+                                                     partition_size, workspace, max_partitions, dtype, stream);
+        if (rc != OPT_GQA_OK) return rc;
+        return opt_gqa_paged_attention_reduce_balanced(out, workspace, context_lens, B, Hq, Hkv, D, partition_size,
+                                                       max_partitions, dtype, stream);
+    }
     float* partial_out = static_cast<float*>(workspace);
     float* partial_lse =
         partial_out ? partial_out + (size_t)(B > 0 ? B : 0) * Hq * (max_partitions > 0 ? max_partitions : 0) * D
@@ -227,7 +276,10 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
 
 size_t opt_gqa_workspace_bytes(int B, int Hq, int D, int max_partitions) {
     if (B <= 0 || Hq <= 0 || D <= 0 || max_partitions <= 0) return 0;
-    return (size_t)B * (size_t)Hq * (size_t)max_partitions * (size_t)(D + 1) * sizeof(float);
+    // Room for either layout: one row per (sequence, head, partition), or the balanced split's pieces (the rows of
+    // up to kBalancedMaxWorkers extra pieces of a group of 8 heads) with its bookkeeping.
+    const size_t rows = (size_t)B * (size_t)Hq * (size_t)max_partitions + (size_t)kBalancedMaxWorkers * 8;
+    return 256 + round_up_256((size_t)B * 16) + round_up_256(rows * 4) + rows * (size_t)D * 4;
 }
 
 int opt_gqa_device_status(void) {

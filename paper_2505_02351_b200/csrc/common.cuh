@@ -141,6 +141,41 @@ int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* 
                      float* partial_out, float* partial_lse, int max_partitions, int* device_status,
                      cudaStream_t stream);
 
+// Workspace of the balanced split (bf16 caches, partition_size > 0).  The stream of 16-token tiles
+// (sequence, KV head, partition order) is cut into one range per worker at TILE granularity; a piece is the
+// part of one partition inside one range, and piece (partition index i in that order, worker w) owns rows
+// (i + w) * G .. + G - 1 of partial_lse / partial_out.  header = {tiles in the stream, workers};
+// seq_info[s] = {tiles, partitions} of one head summed over the sequences before s.
+constexpr int kBalancedMaxWorkers = 2048;
+struct BalancedLayout {
+    size_t header, seq_info, lse, out, total;
+    unsigned long long rows;      // rows of partial_lse / partial_out
+};
+inline size_t round_up_256(size_t x) { return (x + 255) & ~(size_t)255; }
+inline BalancedLayout balanced_layout(int B, int Hq, int Hkv, int D, int max_partitions) {
+    BalancedLayout L;
+    const unsigned long long G = (unsigned long long)(Hq / Hkv);
+    L.rows = ((unsigned long long)B * Hkv * max_partitions + kBalancedMaxWorkers) * G;
+    L.header = 0;
+    L.seq_info = 256;
+    L.lse = L.seq_info + round_up_256((size_t)B * 16);
+    L.out = L.lse + round_up_256((size_t)L.rows * 4);
+    L.total = L.out + (size_t)L.rows * D * 4;
+    return L;
+}
+
+// bf16, partition_size > 0: persistent streaming kernel, one worker per warp (decode_stream.cu).
+// workspace == nullptr writes one partial per partition to partial_out / partial_lse; otherwise the balanced split.
+int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                         int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
+                         int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                         float* partial_out, float* partial_lse, void* workspace, int max_partitions,
+                         int* device_status, cudaStream_t stream);
+
+// Merge of the balanced split's pieces (reduce.cu).
+int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
+                           int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream);
+
 int launch_reduce(void* out, const float* partial_out, const float* partial_lse, const int32_t* context_lens,
                   int B, int Hq, int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream);
 

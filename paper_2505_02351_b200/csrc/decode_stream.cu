@@ -1,0 +1,635 @@
+// Partitioned paged GQA-ALiBi decode attention for bf16 caches on sm_100a, persistent
+// streaming form (Algorithm 2, "Compute context attention with caches"; Eq. 3-5; the
+// long-sequence partitioning described before Eq. 1).
+//
+// Work items are (sequence, KV head, context partition) triples, each producing one
+// normalised partial result and its log-sum-exp for all G query heads of the group
+// ("Shared Key-Value": a K/V tile is brought on-chip once for the whole group).  The
+// grid is persistent: every warp is an independent worker with a private ring of
+// 16-token K/V tiles fetched by 2-D TMA (128-byte swizzle).  The items, laid end to
+// end in (sequence, KV head, partition) order and measured in tiles, are cut into one
+// contiguous range per worker; a worker owns the items that start inside its range and
+// streams them back to back, so the ring never drains between items: page ids, the
+// query rows and the slopes of the next item are fetched while the current one is
+// still being consumed.  The cut is computed by every warp from context_lens alone
+// (two coalesced passes), so there is no scheduler state in global memory.
+//
+// Per tile the warp computes, transposed so that the 16 tokens are the rows and the
+// (up to 8) heads of the group the columns of an m16n8k16 tile,
+//   S^T = K q^T              8 k-steps over the head dimension          (Eq. 3, dot products)
+//   s   = S^T * scale*log2e + slope_h*log2e*(j - (n-1))                 (Eq. 3, ALiBi bias)
+//   running max / denominator per head, p = 2^(s - m) rounded to bf16   (Eq. 4, online)
+//   O^T += V^T p^T           one m16n8k16 per 16 output dims            (Eq. 5)
+// p^T reaches its operand layout through movmatrix; the denominator sums the same
+// rounded p that the tensor core multiplies; accumulation is fp32.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace optgqa {
+
+namespace {
+
+#ifndef OPT_GQA_STREAM_WARPS
+#define OPT_GQA_STREAM_WARPS 4
+#endif
+#ifndef OPT_GQA_STREAM_STAGES
+#define OPT_GQA_STREAM_STAGES 2
+#endif
+#ifndef OPT_GQA_STREAM_CTAS
+#define OPT_GQA_STREAM_CTAS 3
+#endif
+constexpr int kTileTok = 16;                     // tokens per tile (one ring stage holds a K tile and a V tile)
+constexpr int kWarps = OPT_GQA_STREAM_WARPS;     // workers per CTA
+constexpr int kStages = OPT_GQA_STREAM_STAGES;   // ring depth per worker
+constexpr int kCtasPerSm = OPT_GQA_STREAM_CTAS;
+constexpr int kDescSlots = 4;                    // item descriptors a worker keeps (>= items between prefetch and use)
+constexpr unsigned kFull = 0xffffffffu;
+
+struct StreamParams {
+    const __nv_bfloat16* q;
+    const int32_t* block_tables;
+    const int32_t* context_lens;
+    const float* slopes;
+    float* partial_out;
+    float* partial_lse;
+    long long* header;      // balanced split: {tiles in the stream, workers}
+    long long* seq_info;    // balanced split: per sequence {tiles, partitions} of one head over the earlier sequences
+    int* status;
+    float scale;
+    int B;
+    int max_blocks;
+    int Hq;
+    int Hkv;
+    int bs;
+    int partition_size;
+    int max_partitions;
+};
+
+template <int D>
+struct StreamCfg {
+    static constexpr int NBOX = D / 64;                   // 128-byte-wide boxes per token row
+    static constexpr int BOX_BYTES = kTileTok * 128;      // 16 rows x 128 B
+    static constexpr int TILE_BYTES = NBOX * BOX_BYTES;   // K (or V) bytes per tile
+    static constexpr int WARP_RING = kStages * 2 * TILE_BYTES;
+    static constexpr int OFF_DESC = kWarps * WARP_RING;
+    static constexpr int OFF_BAR = OFF_DESC + kWarps * kDescSlots * 32;
+    static constexpr int SMEM = OFF_BAR + kWarps * kStages * 8 + 1024;   // + slack to align the ring to 1 KB
+};
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+// Transposes an 8x8 matrix of 16-bit elements held one row pair per thread (the ldmatrix layout).
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
+// d += a * b, m16n8k16, bf16 operands, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Byte offset of 16-byte chunk `chunk` (0 .. D/8-1) of token row `row` inside a tile stored as
+// NBOX boxes of 16 rows x 128 B with the 128-byte swizzle (chunk index XOR row mod 8).
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+    return (uint32_t)((chunk >> 3) * (kTileTok * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+__device__ __forceinline__ float group_max(float v) {     // over the 8 lanes that share lane & 3
+    v = fmaxf(v, __shfl_xor_sync(kFull, v, 4));
+    v = fmaxf(v, __shfl_xor_sync(kFull, v, 8));
+    return fmaxf(v, __shfl_xor_sync(kFull, v, 16));
+}
+
+__device__ __forceinline__ float group_sum(float v) {
+    v += __shfl_xor_sync(kFull, v, 4);
+    v += __shfl_xor_sync(kFull, v, 8);
+    return v + __shfl_xor_sync(kFull, v, 16);
+}
+
+// Position in the tile stream: streams (sequence, KV head) follow one another in that order, each
+// ceil(n / 16) tiles long; sequences without tokens take no room.
+struct StreamCursor {
+    int s, kvh, n;          // sequence, KV head, context length of s
+    int tiles, parts;       // tiles and partitions of one stream of s
+    int jt;                 // tile inside the stream
+    long long pos;          // the same position in the end-to-end numbering
+    long long tiles_before; // sum of `tiles` over earlier sequences (one head)
+    long long parts_before; // sum of `parts` over earlier sequences (one head)
+};
+
+template <int D, int G, bool kBalanced>
+__global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
+decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                     const StreamParams p) {
+    using C = StreamCfg<D>;
+    constexpr int KS = D / 16;    // k-steps of K q^T
+    constexpr int MT = D / 16;    // m-tiles of V^T p^T
+    extern __shared__ char smem_raw[];
+    char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+
+    grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int P = p.partition_size, P16 = P / kTileTok;    // tiles per full partition
+    const int* __restrict__ lens = p.context_lens;         // an input of the step: not written by the preceding grid
+    if (lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    }
+
+    // ------------------------------------------------------------------ this worker's range of the tile stream
+    long long total = 0;
+    for (int s0 = 0; s0 < p.B; s0 += 32) {
+        const int n = s0 + lane < p.B ? __ldg(lens + s0 + lane) : 0;
+        int tl = (n + kTileTok - 1) / kTileTok;
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) tl += __shfl_xor_sync(kFull, tl, o);
+        total += tl;
+    }
+    total *= p.Hkv;
+    // Never more workers than tiles, so that every worker's range holds at least one tile.
+    const long long grid_workers = (long long)gridDim.x * kWarps, me = (long long)blockIdx.x * kWarps + warp;
+    const long long workers = total < grid_workers ? (total > 0 ? total : 1) : grid_workers;
+    if (kBalanced && me == 0) {
+        grid_dependency_wait();     // the previous reader of the workspace must be done
+        if (lane == 0) {
+            p.header[0] = total;
+            p.header[1] = workers;
+        }
+    }
+    if (total == 0 || me >= workers) return;
+    const long long lo = total * me / workers, hi = total * (me + 1) / workers;
+
+    StreamCursor cur;       // the next piece to be described (runs one piece ahead of the issue side)
+    {
+        // sequence whose tiles contain position lo
+        long long acc_t = 0, acc_p = 0;
+        cur.s = -1;
+        for (int s0 = 0; s0 < p.B && cur.s < 0; s0 += 32) {
+            const int n = s0 + lane < p.B ? __ldg(lens + s0 + lane) : 0;
+            const int tl = (n + kTileTok - 1) / kTileTok, np = (n + P - 1) / P;
+            int incl_t = tl, incl_p = np;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int vt = __shfl_up_sync(kFull, incl_t, o), vp = __shfl_up_sync(kFull, incl_p, o);
+                if (lane >= o) {
+                    incl_t += vt;
+                    incl_p += vp;
+                }
+            }
+            const unsigned hit = __ballot_sync(kFull, (acc_t + incl_t) * p.Hkv > lo);
+            if (hit) {
+                const int src = __ffs(hit) - 1;
+                cur.s = s0 + src;
+                cur.n = __shfl_sync(kFull, n, src);
+                cur.tiles = __shfl_sync(kFull, tl, src);
+                cur.parts = __shfl_sync(kFull, np, src);
+                cur.tiles_before = acc_t + __shfl_sync(kFull, incl_t, src) - cur.tiles;
+                cur.parts_before = acc_p + __shfl_sync(kFull, incl_p, src) - cur.parts;
+            } else {
+                acc_t += __shfl_sync(kFull, incl_t, 31);
+                acc_p += __shfl_sync(kFull, incl_p, 31);
+            }
+        }
+        if (cur.s < 0) return;                               // cannot happen: lo < total
+        const int r = (int)(lo - cur.tiles_before * p.Hkv);
+        cur.kvh = r / cur.tiles;
+        cur.jt = r - cur.kvh * cur.tiles;
+        cur.pos = lo;
+    }
+    auto next_stream = [&]() {
+        cur.jt = 0;
+        if (++cur.kvh == p.Hkv) {
+            cur.kvh = 0;
+            cur.tiles_before += cur.tiles;
+            cur.parts_before += cur.parts;
+            do {
+                ++cur.s;
+                cur.n = cur.s < p.B ? __ldg(lens + cur.s) : 0;
+            } while (cur.s < p.B && cur.n == 0);
+            cur.tiles = (cur.n + kTileTok - 1) / kTileTok;
+            cur.parts = (cur.n + P - 1) / P;
+        }
+    };
+    if (!kBalanced && cur.jt % P16 != 0) {
+        // whole partitions only: the first one that starts at or after lo
+        const int adv = min(P16 - cur.jt % P16, cur.tiles - cur.jt);
+        cur.jt += adv;
+        cur.pos += adv;
+        if (cur.jt == cur.tiles) next_stream();
+    }
+    auto cur_valid = [&]() { return cur.s < p.B && cur.pos < hi; };
+    if (!cur_valid()) return;
+
+    char* ring = smem + warp * C::WARP_RING;
+    int4* desc = reinterpret_cast<int4*>(smem + C::OFF_DESC) + warp * (2 * kDescSlots);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR) + warp * kStages;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < kStages; ++i) mbar_init(&bars[i], 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+
+    // Describes the piece under `cur` in slot (piece & 3), starts the loads of its first 32 page ids, moves `cur`
+    // on.  A piece is the part of one partition that lies inside this worker's range (kBalanced) or one whole
+    // partition (otherwise).  desc[2i] = {s, kvh, n, first tile in the stream}, desc[2i+1] = {tiles, row of the
+    // partial result of the group's first head}.
+    int pieces = 0;               // pieces described so far
+    int pages_nxt = 0;            // lane l: physical page of tile l of the piece described last
+    auto describe_next = [&]() {
+        const int part = cur.jt / P16;
+        int len = min((part + 1) * P16, cur.tiles) - cur.jt;
+        int obase;
+        if (kBalanced) {
+            len = (int)min((long long)len, hi - cur.pos);
+            // pieces are numbered by (partition index in the end-to-end order) + (worker index): both only grow
+            obase = (int)((cur.parts_before * p.Hkv + (long long)cur.kvh * cur.parts + part + me) * G);
+            if (lane == 0 && cur.kvh == 0 && cur.jt == 0) {
+                p.seq_info[2 * cur.s] = cur.tiles_before;
+                p.seq_info[2 * cur.s + 1] = cur.parts_before;
+            }
+            // Where this range and a partition end together inside a stream, the next piece is two numbers on:
+            // mark the number in between as empty, so that the merge can sweep the stream's numbers without gaps.
+            if (cur.pos + len == hi && cur.jt + len < cur.tiles && (cur.jt + len) % P16 == 0 && lane < G)
+                p.partial_lse[obase + G + lane] = -INFINITY;
+        } else {
+            obase = (cur.s * p.Hq + cur.kvh * G) * p.max_partitions + part;
+        }
+        if (lane == 0) {
+            desc[2 * (pieces & (kDescSlots - 1))] = make_int4(cur.s, cur.kvh, cur.n, cur.jt);
+            desc[2 * (pieces & (kDescSlots - 1)) + 1] = make_int4(len, obase, 0, 0);
+        }
+        const int tok = (cur.jt + lane) * kTileTok;
+        pages_nxt = lane < len ? __ldg(p.block_tables + (size_t)cur.s * p.max_blocks + tok / p.bs) : 0;
+        ++pieces;
+        cur.pos += len;
+        cur.jt += len;
+        if (cur.jt == cur.tiles) next_stream();
+        __syncwarp();
+    };
+
+    // ------------------------------------------------------------------ issue side
+    int is_piece = -1, is_j = 0, is_ntile = 0, is_kvh = 0, is_tile0 = 0, is_s = 0;
+    int pages_cur = 0;
+    uint32_t issued = 0, consumed = 0;     // tiles over the worker's whole stream: ring slot = count % kStages
+    int cs_piece = -1;
+    // B fragments of q for the piece entered last on the issue side (rows = heads; heads >= G are zero), its slopes
+    uint32_t q_nxt[KS][2];
+    float sl_nxt[2];
+    const float qscale = p.scale * kLog2e;
+
+    auto issue_one = [&]() {               // precondition: a tile may be issued
+        if (is_j == is_ntile) {
+            // enter the next piece: its descriptor and first page ids were produced one piece ago
+            ++is_piece;
+            const int4 d0 = desc[2 * (is_piece & (kDescSlots - 1))];
+            is_ntile = desc[2 * (is_piece & (kDescSlots - 1)) + 1].x;
+            pages_cur = pages_nxt;
+            is_j = 0;
+            is_s = d0.x;
+            is_kvh = d0.y;
+            is_tile0 = d0.w;
+            const uint32_t* qh = reinterpret_cast<const uint32_t*>(
+                p.q + ((size_t)d0.x * p.Hq + (size_t)d0.y * G + (g < G ? g : 0)) * D);
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                q_nxt[ks][0] = g < G ? __ldg(qh + ks * 8 + t) : 0u;
+                q_nxt[ks][1] = g < G ? __ldg(qh + ks * 8 + 4 + t) : 0u;
+            }
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+                sl_nxt[c] = (p.slopes && 2 * t + c < G) ? __ldg(p.slopes + d0.y * G + 2 * t + c) * kLog2e : 0.f;
+            if (cur_valid()) describe_next();
+        } else if ((is_j & 31) == 0) {
+            // pieces longer than 512 tokens: the next 32 page ids
+            const int tok = (is_tile0 + is_j + lane) * kTileTok;
+            pages_cur = is_j + lane < is_ntile ? __ldg(p.block_tables + (size_t)is_s * p.max_blocks + tok / p.bs) : 0;
+        }
+        const int phys = __shfl_sync(kFull, pages_cur, is_j & 31);
+        if (lane == 0) {
+            const int tok = (is_tile0 + is_j) * kTileTok;
+            const int row = (phys * p.Hkv + is_kvh) * p.bs + tok % p.bs;       // row of the [rows, D] view
+            const int st = issued % kStages;
+            char* dst = ring + st * 2 * C::TILE_BYTES;
+            mbar_expect_tx(&bars[st], 2 * C::TILE_BYTES);
+#pragma unroll
+            for (int b = 0; b < C::NBOX; ++b) {
+                tma_load_2d(dst + b * C::BOX_BYTES, &map_k, b * 64, row, &bars[st]);
+                tma_load_2d(dst + C::TILE_BYTES + b * C::BOX_BYTES, &map_v, b * 64, row, &bars[st]);
+            }
+        }
+        ++is_j;
+        ++issued;
+    };
+    // A tile may be issued while a ring slot is free and there is a tile left; a new piece is entered only
+    // once the consume side has entered the one before it (q_nxt / sl_nxt hold one piece).
+    auto issue_allowed = [&]() {
+        if (issued - consumed >= (uint32_t)kStages) return false;
+        if (is_j < is_ntile) return true;
+        return is_piece < pieces - 1 && is_piece <= cs_piece;
+    };
+
+    grid_dependency_wait();     // the cache may still be receiving this step's appended tokens
+    describe_next();            // piece 0
+    while (issue_allowed()) issue_one();
+
+    // ------------------------------------------------------------------ consume side
+    uint32_t qb[KS][2];
+    float sl[2] = {0.f, 0.f};
+    float o[MT][4];
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    int cs_j = 0, cs_ntile = 0, cs_n = 0, cs_tile0 = 0, cs_obase = 0;
+    const int ostride = kBalanced ? 1 : p.max_partitions;     // distance between the rows of consecutive heads
+    const int lrow = lane & 7, lmat = lane >> 3;
+    bool ok = true;
+
+    while (consumed != issued) {
+        if (cs_j == cs_ntile) {
+            // enter the next piece
+            ++cs_piece;
+            const int4 d0 = desc[2 * (cs_piece & (kDescSlots - 1))], d1 = desc[2 * (cs_piece & (kDescSlots - 1)) + 1];
+            cs_n = d0.z;
+            cs_tile0 = d0.w;
+            cs_ntile = d1.x;
+            cs_obase = d1.y;
+            cs_j = 0;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                qb[ks][0] = q_nxt[ks][0];
+                qb[ks][1] = q_nxt[ks][1];
+            }
+            sl[0] = sl_nxt[0];
+            sl[1] = sl_nxt[1];
+#pragma unroll
+            for (int i = 0; i < MT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+            m0 = m1 = -INFINITY;
+            l0 = l1 = 0.f;
+        }
+        const int st = consumed % kStages;
+        char* kst = ring + st * 2 * C::TILE_BYTES;
+        char* vst = kst + C::TILE_BYTES;
+        ok = __all_sync(kFull, mbar_wait(&bars[st], (consumed / kStages) & 1, p.status));
+        if (!ok) break;
+
+        const int j0 = (cs_tile0 + cs_j) * kTileTok;
+        const int valid = min(kTileTok, cs_n - j0);
+        if (valid < kTileTok) {
+            // Rows past the end of the sequence hold whatever the page held: zero the V rows so that
+            // 0 * garbage cannot produce NaN (their scores are masked below).
+            for (int r = valid + (lane >> 3); r < kTileTok; r += 4)
+#pragma unroll
+                for (int b = 0; b < C::NBOX; ++b)
+                    *reinterpret_cast<uint4*>(vst + b * C::BOX_BYTES + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+            __syncwarp();
+        }
+
+        // ---- S^T[token][head]: rows = the tile's 16 tokens, columns = heads of the group
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+            const uint32_t kbase = smem_u32(kst);
+            const int krow = lrow + 8 * (lmat & 1);          // matrices 0,2: tokens 0-7; 1,3: tokens 8-15
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t a[4];
+                ldmatrix_x4(a, kbase + swz(krow, 2 * ks + (lmat >> 1)));
+                mma_bf16(sc, a, qb[ks][0], qb[ks][1]);
+            }
+        }
+        // thread holds tokens j0 + g (sc[0], sc[1]) and j0 + g + 8 (sc[2], sc[3]) for heads 2t, 2t + 1
+        {
+            const int ja = j0 + g;
+            const float relA = (float)(ja - (cs_n - 1)), relB = relA + 8.f;
+            sc[0] = fmaf(sc[0], qscale, sl[0] * relA);
+            sc[1] = fmaf(sc[1], qscale, sl[1] * relA);
+            sc[2] = fmaf(sc[2], qscale, sl[0] * relB);
+            sc[3] = fmaf(sc[3], qscale, sl[1] * relB);
+            if (ja >= cs_n) sc[0] = sc[1] = -INFINITY;
+            if (ja + 8 >= cs_n) sc[2] = sc[3] = -INFINITY;
+        }
+        const float m0n = fmaxf(m0, group_max(fmaxf(sc[0], sc[2])));
+        const float m1n = fmaxf(m1, group_max(fmaxf(sc[1], sc[3])));
+        const float a0 = ex2(m0 - m0n), a1 = ex2(m1 - m1n);
+        const bool rescale = __any_sync(kFull, m0n > m0 || m1n > m1);
+        m0 = m0n;
+        m1 = m1n;
+        // p rounded to bf16 once: the same values feed the tensor core and the denominator
+        const __nv_bfloat162 pa = __floats2bfloat162_rn(ex2(sc[0] - m0n), ex2(sc[1] - m1n));   // token g
+        const __nv_bfloat162 pb = __floats2bfloat162_rn(ex2(sc[2] - m0n), ex2(sc[3] - m1n));   // token g + 8
+        const float2 fa = __bfloat1622float2(pa), fb = __bfloat1622float2(pb);
+        l0 = fmaf(l0, a0, fa.x + fb.x);
+        l1 = fmaf(l1, a1, fa.y + fb.y);
+        const uint32_t b0 = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pa));   // tokens 2t, 2t+1 of head g
+        const uint32_t b1 = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pb));   // tokens 2t+8, 2t+9
+        if (rescale) {
+#pragma unroll
+            for (int i = 0; i < MT; ++i) {
+                o[i][0] *= a0;
+                o[i][1] *= a1;
+                o[i][2] *= a0;
+                o[i][3] *= a1;
+            }
+        }
+
+        // ---- O^T[dim][head] += V^T[dim][token] * p^T[token][head]; V transposed on the fly by ldmatrix.trans
+        {
+            const uint32_t vbase = smem_u32(vst);
+            const int vrow = lrow + 8 * (lmat >> 1);         // matrices 0,1: tokens 0-7; 2,3: tokens 8-15
+#pragma unroll
+            for (int i = 0; i < MT; ++i) {
+                uint32_t a[4];
+                ldmatrix_x4_trans(a, vbase + swz(vrow, 2 * i + (lmat & 1)));
+                mma_bf16(o[i], a, b0, b1);
+            }
+        }
+        ++cs_j;
+        ++consumed;
+
+        if (cs_j == cs_ntile) {
+            // ---- the piece is complete: normalise, write the partial result and its log-sum-exp
+            const float L0 = group_sum(l0), L1 = group_sum(l1);
+            const float i0 = 1.f / L0, i1 = 1.f / L1;
+            if (2 * t < G) {
+                const size_t row = (size_t)cs_obase + (size_t)(2 * t) * ostride;
+                float* po = p.partial_out + row * D;
+#pragma unroll
+                for (int i = 0; i < MT; ++i) {
+                    po[16 * i + g] = o[i][0] * i0;
+                    po[16 * i + 8 + g] = o[i][2] * i0;
+                }
+                if (g == 0) p.partial_lse[row] = (m0 + lg2(L0)) * kLn2;
+            }
+            if (2 * t + 1 < G) {
+                const size_t row = (size_t)cs_obase + (size_t)(2 * t + 1) * ostride;
+                float* po = p.partial_out + row * D;
+#pragma unroll
+                for (int i = 0; i < MT; ++i) {
+                    po[16 * i + g] = o[i][1] * i1;
+                    po[16 * i + 8 + g] = o[i][3] * i1;
+                }
+                if (g == 0) p.partial_lse[row] = (m1 + lg2(L1)) * kLn2;
+            }
+        }
+
+        // The slot just consumed may have been written by this warp (the zeroed rows): order those
+        // generic-proxy writes before the async-proxy copy that refills it.
+        fence_proxy_async();
+        __syncwarp();
+        while (issue_allowed()) issue_one();
+    }
+
+    if (!ok) {
+        // A wait gave up (already recorded).  Give the copies still in flight one more bounded
+        // chance to land before this CTA's shared memory is released.
+        for (uint32_t kk = consumed; kk != issued; ++kk) mbar_wait(&bars[kk % kStages], (kk / kStages) & 1, p.status);
+    }
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// The cache seen as a 2-D bf16 tensor [num_blocks*Hkv*bs rows, D]; a box is 16 token rows x 64 dims (128 B).
+bool make_map(CUtensorMap* map, const void* cache, uint64_t rows, int D) {
+    EncodeFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTileTok};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int counts[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!counts[dev] && cudaDeviceGetAttribute(&counts[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return counts[dev];
+}
+
+template <int D, int G, bool kBalanced>
+int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams& p, cudaStream_t stream) {
+    using C = StreamCfg<D>;
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    if (dev < 64 && !configured[dev]) {
+        if (cudaFuncSetAttribute(decode_stream_kernel<D, G, kBalanced>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 C::SMEM) != cudaSuccess)
+            return OPT_GQA_ERR_CUDA;
+        configured[dev] = true;
+    }
+    const int sms = sm_count();
+    if (sms <= 0) return OPT_GQA_ERR_CUDA;
+    // One resident wave; never more workers than there could be partitions, nor than the workspace has room for.
+    const long long items = (long long)p.B * p.Hkv * p.max_partitions;
+    long long ctas = (items + kWarps - 1) / kWarps;
+    if (ctas > (long long)sms * kCtasPerSm) ctas = (long long)sms * kCtasPerSm;
+    if (ctas > kBalancedMaxWorkers / kWarps) ctas = kBalancedMaxWorkers / kWarps;
+    return launch_dependent(decode_stream_kernel<D, G, kBalanced>, dim3((unsigned)ctas), dim3(kWarps * 32), C::SMEM,
+                            stream, mk, mv, p);
+}
+
+template <int D, bool kBalanced>
+int launch_g(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams& p, int G, cudaStream_t stream) {
+    switch (G) {
+        case 1: return launch_one<D, 1, kBalanced>(mk, mv, p, stream);
+        case 2: return launch_one<D, 2, kBalanced>(mk, mv, p, stream);
+        case 4: return launch_one<D, 4, kBalanced>(mk, mv, p, stream);
+        case 8: return launch_one<D, 8, kBalanced>(mk, mv, p, stream);
+    }
+    return OPT_GQA_ERR_SHAPE;
+}
+
+}  // namespace
+
+// workspace == nullptr: one partial result per partition in partial_out / partial_lse ([B, Hq, max_partitions, ...]).
+// Otherwise the balanced split: pieces and bookkeeping go to `workspace` (see balanced_layout).
+int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                         int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
+                         int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                         float* partial_out, float* partial_lse, void* workspace, int max_partitions,
+                         int* device_status, cudaStream_t stream) {
+    const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
+    if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
+    CUtensorMap mk, mv;
+    if (!make_map(&mk, k_cache, rows, D) || !make_map(&mv, v_cache, rows, D)) return OPT_GQA_ERR_CUDA;
+    StreamParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.block_tables = block_tables;
+    p.context_lens = context_lens;
+    p.slopes = alibi_slopes;
+    p.partial_out = partial_out;
+    p.partial_lse = partial_lse;
+    p.header = nullptr;
+    p.seq_info = nullptr;
+    if (workspace) {
+        const BalancedLayout L = balanced_layout(B, Hq, Hkv, D, max_partitions);
+        if (L.rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
+        char* ws = static_cast<char*>(workspace);
+        p.header = reinterpret_cast<long long*>(ws + L.header);
+        p.seq_info = reinterpret_cast<long long*>(ws + L.seq_info);
+        p.partial_lse = reinterpret_cast<float*>(ws + L.lse);
+        p.partial_out = reinterpret_cast<float*>(ws + L.out);
+    }
+    p.status = device_status;
+    p.scale = scale;
+    p.B = B;
+    p.max_blocks = max_blocks_per_seq;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.bs = bs;
+    p.partition_size = partition_size;
+    p.max_partitions = max_partitions;
+    const int G = Hq / Hkv;
+    if (workspace) {
+        if (D == 128) return launch_g<128, true>(mk, mv, p, G, stream);
+        if (D == 64) return launch_g<64, true>(mk, mv, p, G, stream);
+    } else {
+        if (D == 128) return launch_g<128, false>(mk, mv, p, G, stream);
+        if (D == 64) return launch_g<64, false>(mk, mv, p, G, stream);
+    }
+    return OPT_GQA_ERR_SHAPE;
+}
+
+}  // namespace optgqa

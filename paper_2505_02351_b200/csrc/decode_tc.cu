@@ -23,9 +23,19 @@ namespace optgqa {
 
 namespace {
 
-constexpr int kTileTok = 16;   // tokens per tile (one ring stage holds a K tile and a V tile)
-constexpr int kWarps = 4;      // warps per CTA, each with a private ring
-constexpr int kStages = 2;     // ring depth per warp
+#ifndef OPT_GQA_TC_WARPS
+#define OPT_GQA_TC_WARPS 4
+#endif
+#ifndef OPT_GQA_TC_STAGES
+#define OPT_GQA_TC_STAGES 2
+#endif
+#ifndef OPT_GQA_TC_CTAS
+#define OPT_GQA_TC_CTAS 3
+#endif
+constexpr int kTileTok = 16;                 // tokens per tile (one ring stage holds a K tile and a V tile)
+constexpr int kWarps = OPT_GQA_TC_WARPS;     // warps per CTA, each with a private ring
+constexpr int kStages = OPT_GQA_TC_STAGES;   // ring depth per warp
+constexpr int kMinCtas = OPT_GQA_TC_CTAS;    // CTAs per SM the register budget is held to
 constexpr unsigned kFull = 0xffffffffu;
 
 struct TcParams {
@@ -94,7 +104,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 }
 
 template <int D, int G>
-__global__ void __launch_bounds__(kWarps * 32, 3)
+__global__ void __launch_bounds__(kWarps * 32, kMinCtas)
 decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                  const TcParams p) {
     using C = TcCfg<D, G>;

@@ -25,11 +25,11 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
     const int n = context_lens[s];         // an input of the step, not produced by the decode grid
     const int np = (n + partition_size - 1) / partition_size;
     T* o = out + (size_t)row * D;
+    grid_dependency_wait();                // the partials come from the decode grid; out may still be read by its last user
     if (np <= 0) {
         for (int d = threadIdx.x; d < D; d += blockDim.x) o[d] = T(0.f);
         return;
     }
-    grid_dependency_wait();                // the partials come from the decode grid
     const float* lse = partial_lse + (size_t)row * max_partitions;
     const float* po = partial_out + (size_t)row * max_partitions * D + lane * V;
 
@@ -75,6 +75,106 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
     }
 }
 
+// The same merge over the pieces of the balanced split (see balanced_layout).  The pieces of the row's
+// (sequence, KV head) stream carry consecutive numbers -- (partition index) + (worker index), and from one piece
+// to the next exactly one of the two grows, or both, in which case the decode kernel marked the number in between
+// with lse = -inf -- so the merge is one sweep over rows r0 .. r1 of partial_lse / partial_out: r0 belongs to the
+// stream's first tile, r1 to its last.  All loads of the sweep are independent.
+// A CTA has 8 warps and merges 8 / WPR rows, WPR warps per row (chosen by the launcher from the number of
+// rows, so that batches of many short sequences do not pay for warps with nothing to sweep).
+constexpr int kBalWarps = 8;
+
+template <typename T, int D, int WPR>
+__global__ void __launch_bounds__(kBalWarps * 32)
+reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_out,
+                       const float* __restrict__ partial_lse, const long long* __restrict__ header,
+                       const long long* __restrict__ seq_info, const int32_t* __restrict__ context_lens, int rows,
+                       int Hq, int Hkv, int partition_size) {
+    constexpr int V = D / 32;             // columns per lane
+    constexpr int RPB = kBalWarps / WPR;  // rows per CTA
+    __shared__ float s_num[kBalWarps][D];
+    __shared__ float s_den[kBalWarps];
+    __shared__ float s_max[kBalWarps];
+    grid_dependency_launch();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rib = warp / WPR, sub = warp % WPR;
+    const int row = blockIdx.x * RPB + rib;                 // s * Hq + h
+    const bool active = row < rows;
+    const int s = active ? row / Hq : 0, h = active ? row % Hq : 0, G = Hq / Hkv, kvh = h / G, hh = h % G;
+    const int n = active ? context_lens[s] : 0;             // an input of the step, not produced by the decode grid
+    const int np = (n + partition_size - 1) / partition_size;
+    grid_dependency_wait();                                 // the pieces come from the decode grid
+
+    int R = 0;
+    const float* lse = partial_lse;
+    const float* po = partial_out;
+    if (np > 0) {
+        const long long total = header[0], workers = header[1];
+        const int tiles = (n + 15) / 16;
+        const long long first_tile = seq_info[2 * s] * Hkv + (long long)kvh * tiles;
+        const long long first_part = seq_info[2 * s + 1] * Hkv + (long long)kvh * np;
+        // worker whose range [floor(T w / W), floor(T (w + 1) / W)) holds tile x: floor(((x + 1) W - 1) / T)
+        const long long r0 = first_part + ((first_tile + 1) * workers - 1) / total;
+        const long long r1 = first_part + np - 1 + ((first_tile + tiles) * workers - 1) / total;
+        R = (int)(r1 - r0 + 1);
+        lse += (size_t)r0 * G + hh;                          // stride G
+        po += ((size_t)r0 * G + hh) * D + lane * V;          // stride G * D
+    }
+
+    float M = -INFINITY;
+    for (int i = sub * 32 + lane; i < R; i += WPR * 32) M = fmaxf(M, lse[(size_t)i * G]);
+#pragma unroll
+    for (int o2 = 16; o2 >= 1; o2 >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o2));
+    if (WPR > 1) {
+        if (lane == 0) s_max[warp] = M;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < WPR; ++w) M = fmaxf(M, s_max[rib * WPR + w]);
+    }
+
+    float num[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) num[v] = 0.f;
+    float den = 0.f;
+#pragma unroll 4
+    for (int i = sub; i < R; i += WPR) {
+        const float l = lse[(size_t)i * G];
+        const bool piece = l > -INFINITY;                     // false for the empty numbers: their rows hold nothing
+        const float w = piece ? ex2((l - M) * kLog2e) : 0.f;
+        den += w;
+        if constexpr (V == 4) {
+            float4 x = *reinterpret_cast<const float4*>(po + (size_t)i * G * D);
+            if (!piece) x = make_float4(0.f, 0.f, 0.f, 0.f);
+            num[0] = fmaf(w, x.x, num[0]);
+            num[1] = fmaf(w, x.y, num[1]);
+            num[2] = fmaf(w, x.z, num[2]);
+            num[3] = fmaf(w, x.w, num[3]);
+        } else {
+            float2 x = *reinterpret_cast<const float2*>(po + (size_t)i * G * D);
+            if (!piece) x = make_float2(0.f, 0.f);
+            num[0] = fmaf(w, x.x, num[0]);
+            num[1] = fmaf(w, x.y, num[1]);
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) s_num[warp][lane * V + v] = num[v];
+    if (lane == 0) s_den[warp] = den;
+    __syncthreads();
+    if (!active) return;
+    T* o = out + (size_t)row * D;
+    for (int d = sub * 32 + lane; d < D; d += WPR * 32) {
+        float a = 0.f, b = 0.f;
+#pragma unroll
+        for (int w = 0; w < WPR; ++w) {
+            a += s_num[rib * WPR + w][d];
+            b += s_den[rib * WPR + w];
+        }
+        const float r = np > 0 ? a / b : 0.f;                 // an empty sequence gives a zero row
+        if constexpr (sizeof(T) == 2) o[d] = __float2bfloat16_rn(r);
+        else o[d] = r;
+    }
+}
+
 template <typename T, int D>
 static int launch_reduce_t(void* out, const float* partial_out, const float* partial_lse,
                            const int32_t* context_lens, int B, int Hq, int partition_size, int max_partitions,
@@ -98,6 +198,42 @@ int launch_reduce(void* out, const float* partial_out, const float* partial_lse,
                                            max_partitions, stream);
     return launch_reduce_t<float, 64>(out, partial_out, partial_lse, context_lens, B, Hq, partition_size,
                                       max_partitions, stream);
+}
+
+template <typename T, int D, int WPR>
+static int launch_reduce_balanced_w(void* out, const char* ws, const BalancedLayout& L, const int32_t* context_lens,
+                                    int B, int Hq, int Hkv, int partition_size, cudaStream_t stream) {
+    const int rows = B * Hq, rpb = kBalWarps / WPR;
+    return launch_dependent(reduce_balanced_kernel<T, D, WPR>, dim3((unsigned)((rows + rpb - 1) / rpb)),
+                            dim3(kBalWarps * 32), 0, stream, static_cast<T*>(out),
+                            reinterpret_cast<const float*>(ws + L.out), reinterpret_cast<const float*>(ws + L.lse),
+                            reinterpret_cast<const long long*>(ws + L.header),
+                            reinterpret_cast<const long long*>(ws + L.seq_info), context_lens, rows, Hq, Hkv,
+                            partition_size);
+}
+
+template <typename T, int D>
+static int launch_reduce_balanced_t(void* out, const char* ws, const BalancedLayout& L, const int32_t* context_lens,
+                                    int B, int Hq, int Hkv, int partition_size, cudaStream_t stream) {
+    // About 8192 warps in all: 8 per row for a few long rows, 1 per row for batches of many rows.
+    const long long rows = (long long)B * Hq;
+    if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+    if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+    if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+    return launch_reduce_balanced_w<T, D, 1>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+}
+
+int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
+                           int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream) {
+    const BalancedLayout L = balanced_layout(B, Hq, Hkv, D, max_partitions);
+    const char* ws = static_cast<const char*>(workspace);
+    if (dtype == OPT_GQA_BF16) {
+        if (D == 128)
+            return launch_reduce_balanced_t<__nv_bfloat16, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+        return launch_reduce_balanced_t<__nv_bfloat16, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+    }
+    if (D == 128) return launch_reduce_balanced_t<float, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+    return launch_reduce_balanced_t<float, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
 }
 
 }  // namespace optgqa

@@ -41,6 +41,30 @@ def test_config3_long_sequence_partitioned():
     assert wl.partition_size == 512
     _check(wl)
     _check(wl, simt=True)
+    _check(wl, balanced=True)
+
+
+def test_balanced_split_on_the_named_workloads():
+    _check(W.make_config(2, poison=True), partition_size=256, balanced=True)
+    _check(W.make_config(4, poison=True), partition_size=512, balanced=True)
+    _check(W.make_config(4, poison=True), partition_size=1024, balanced=True)
+
+
+def test_decode_step_one_call_matches_the_oracle():
+    """opt_gqa_decode_step (append -> balanced decode -> reduce for bf16; per-partition partials for fp32)."""
+    for wl, P in ((W.make_config(3, shrink=8), 512), (W.make_config(4, poison=True), 512), (W.make_config(1), 32),
+                  (W.make_config(2), 0)):
+        d = util.DeviceWorkload(wl)
+        maxP = max(1, (int(wl.context_lens.max()) + P - 1) // P) if P else 1
+        ws = torch.full((binding.workspace_bytes(wl.B, wl.Hq, wl.D, maxP),), 0xff, device="cuda:0", dtype=torch.uint8)
+        binding.decode_step(d.out, d.q, d.k_new, d.v_new, d.slot_mapping, d.k_cache, d.v_cache, d.block_tables,
+                            d.context_lens, d.alibi_slopes, wl.scale, partition_size=P, workspace=ws if P else None,
+                            max_partitions=maxP)
+        torch.cuda.synchronize()
+        assert binding.device_status() == 0
+        want = util.oracle_attention(wl)
+        got = d.out.double().cpu().numpy()
+        assert np.max(np.abs(got - want)) <= util.TOL[wl.dtype], wl.name
 
 
 def test_config4_ragged_large_batch_with_append():
@@ -59,9 +83,11 @@ def test_shape_matrix(dtype, D, Hq, Hkv, bs):
     _check(wl)
     _check(wl, partition_size=64)
     _check(wl, partition_size=0, slopes=False)
-    if dtype == "bf16":        # the CUDA-core kernel on bf16 caches (fp32 always runs on it)
+    if dtype == "bf16":        # the CUDA-core kernel on bf16 caches (fp32 always runs on it); the balanced split
         _check(wl, simt=True)
         _check(wl, partition_size=64, simt=True)
+        _check(wl, partition_size=64, balanced=True)
+        _check(wl, partition_size=16, balanced=True, slopes=False)
 
 
 @pytest.mark.parametrize("P", [16, 48, 512, 4096])
@@ -69,6 +95,17 @@ def test_any_partition_size_agrees_with_single_pass(P):
     wl = W.make_custom("p", "bf16", 8, 2, 128, 16, [700, 33, 2049], seed=21)
     _check(wl, partition_size=P)
     _check(wl, partition_size=P, simt=True)
+    _check(wl, partition_size=P, balanced=True)
+
+
+def test_balanced_split_with_fewer_tiles_than_workers_and_empty_sequences():
+    # 3 + 1 + 0 + 2 tiles per head: most workers of the persistent grid get an empty range
+    wl = W.make_custom("few", "bf16", 8, 2, 128, 16, [40, 7, 0, 32], seed=25, poison=True)
+    _check(wl, partition_size=16, balanced=True)
+    _check(wl, partition_size=512, balanced=True)
+    wl0 = W.make_custom("none", "bf16", 8, 2, 128, 16, [0, 0], seed=26)
+    got, _ = util.gpu_decode(wl0, partition_size=64, balanced=True)
+    assert np.array_equal(got, np.zeros_like(got))
 
 
 def test_partials_match_the_oracle_partials():

@@ -22,13 +22,26 @@ class DeviceWorkload:
         self.out = torch.full_like(self.q, float("nan"))
 
 
-def gpu_decode(wl: W.Workload, partition_size=None, append=True, slopes=True, simt=False):
-    """append + decode (+ reduce) through the C ABI; returns (out float64 numpy, DeviceWorkload)."""
+def gpu_decode(wl: W.Workload, partition_size=None, append=True, slopes=True, simt=False, balanced=False):
+    """append + decode (+ reduce) through the C ABI; returns (out float64 numpy, DeviceWorkload).
+
+    balanced=True takes the load-balanced split (decode_balanced + reduce_balanced, bf16, partition_size > 0)."""
     d = DeviceWorkload(wl)
     P = wl.partition_size if partition_size is None else partition_size
     if append:
         binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
     sl = d.alibi_slopes if slopes else None
+    if balanced:
+        assert P > 0 and wl.dtype == "bf16"
+        maxP = max(1, (int(wl.context_lens.max()) + P - 1) // P) if wl.B else 1
+        ws = torch.full((binding.workspace_bytes(max(wl.B, 1), wl.Hq, wl.D, maxP) // 4,), float("nan"), device="cuda:0",
+                        dtype=torch.float32)
+        binding.paged_attention_decode_balanced(d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, sl, wl.scale,
+                                                P, ws, maxP)
+        binding.paged_attention_reduce_balanced(d.out, ws, d.context_lens, wl.Hkv, P, maxP)
+        torch.cuda.synchronize()
+        assert binding.device_status() == 0
+        return d.out.double().cpu().numpy(), d
     decode = binding.paged_attention_decode_simt if simt else binding.paged_attention_decode
     if P > 0:
         maxP = max(1, (int(wl.context_lens.max()) + P - 1) // P) if wl.B else 1
@@ -56,7 +69,7 @@ def oracle_inputs(wl: W.Workload, append=True):
                 qsl=None if wl.q_start_loc is None else wl.q_start_loc.numpy())
 
 
-def oracle_attention(wl: W.Workload, append=True, slopes=True, simt=False):
+def oracle_attention(wl: W.Workload, append=True, slopes=True, simt=False, balanced=False):
     a = oracle_inputs(wl, append)
     return oracle.paged_attention(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"] if slopes else None, wl.scale,
                                   wl.dtype, q_start_loc=a["qsl"])
