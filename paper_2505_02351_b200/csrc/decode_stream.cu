@@ -37,7 +37,7 @@ namespace {
 #define OPT_GQA_STREAM_STAGES 2
 #endif
 #ifndef OPT_GQA_STREAM_CTAS
-#define OPT_GQA_STREAM_CTAS 3
+#define OPT_GQA_STREAM_CTAS 2
 #endif
 constexpr int kTileTok = 16;                     // tokens per tile (one ring stage holds a K tile and a V tile)
 constexpr int kWarps = OPT_GQA_STREAM_WARPS;     // workers per CTA
