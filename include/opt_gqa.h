@@ -54,6 +54,10 @@ extern "C" {
 #define OPT_GQA_ERR_ALIGN (-4)   /* a data pointer is not 16-byte aligned                 */
 #define OPT_GQA_ERR_CUDA (-5)    /* the CUDA runtime refused the launch or a copy         */
 #define OPT_GQA_ERR_TIMEOUT (-6) /* a bounded device-side wait ran out (device status)    */
+#define OPT_GQA_ERR_SCRATCH (-7) /* the call needs more than OPT_GQA_STATIC_SCRATCH_BYTES  */
+
+/* Size of the scratch array built into the library for opt_gqa_paged_attention_decode_no_alloc. */
+#define OPT_GQA_STATIC_SCRATCH_BYTES (8u << 20)
 
 /*
  * Slot-mapped write of new tokens' K/V into the paged cache: Algorithm 1,
@@ -163,6 +167,34 @@ int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, co
 int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const float* partial_lse,
                                    const int32_t* context_lens, int B, int Hq, int D, int partition_size,
                                    int max_partitions, int dtype, void* stream);
+
+/*
+ * Partitioned decode and merge in one call, for callers that cannot provide a
+ * workspace.  (The paper has no counterpart: this is a packaging variant of the two
+ * calls above.)  Some hosts of the library cannot allocate device memory where they
+ * call it -- code running inside an engine that has already given all free memory to
+ * the cache pool, or in a callback where cudaMalloc is off limits because it
+ * synchronises the device.  This entry point allocates nothing, neither on the host nor
+ * on the device: the partitions' partial results go to a fixed array of
+ * OPT_GQA_STATIC_SCRATCH_BYTES (8 MiB) that is part of the loaded library.
+ *
+ * Result: the same out [B, Hq, D] as opt_gqa_paged_attention_decode with partition_size
+ * = P > 0 followed by opt_gqa_paged_attention_reduce; arguments as there.
+ *
+ *  - Limit: B * Hq * max_partitions * (D + 1) * 4 bytes must fit in the array;
+ *    otherwise OPT_GQA_ERR_SCRATCH is returned and nothing is enqueued.
+ *  - The array exists once per GPU, from the first use of the library on that GPU until
+ *    the process exits, and all calls on that GPU share it: calls that can overlap on the
+ *    GPU (different streams, no ordering between them) race on it.  It needs no clearing;
+ *    what a previous call left in it is never read.
+ *  - The first call on each device looks up the array's device address (a runtime call
+ *    made with that device current); make that first call outside any stream capture.
+ */
+int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                            const int32_t* block_tables, int max_blocks_per_seq,
+                                            const int32_t* context_lens, const float* alibi_slopes, float scale,
+                                            int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                                            int partition_size, int max_partitions, int dtype, void* stream);
 
 /*
  * Multi-token (chunked-prefill) variant on tensor cores: the prompt branch of

@@ -32,6 +32,8 @@ SIGNATURES = {
     "opt_gqa_paged_attention_decode_balanced": (_i, [_vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                                      _i, _vp, _i, _i, _vp]),
     "opt_gqa_paged_attention_reduce_balanced": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp]),
+    "opt_gqa_paged_attention_decode_no_alloc": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i,
+                                                     _i64, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_reduce": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_prefill": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i,
                                              _i, _i64, _i, _vp]),
@@ -155,6 +157,19 @@ def paged_attention_reduce_balanced(out, workspace, context_lens, Hkv: int, part
     _check(load().opt_gqa_paged_attention_reduce_balanced(
         _ptr(out), _ptr(workspace), _ptr(context_lens), B, Hq, Hkv, D, partition_size, max_partitions,
         _DTYPE_CODE[out.dtype], _stream(stream)), "opt_gqa_paged_attention_reduce_balanced")
+
+
+def paged_attention_decode_no_alloc(out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
+                                    partition_size: int, max_partitions: int, stream=None) -> None:
+    """Partitioned decode + merge with the library's built-in scratch array (nothing is allocated)."""
+    B, Hq, D = q.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    assert block_tables.dtype == torch.int32 and context_lens.dtype == torch.int32
+    assert alibi_slopes is None or alibi_slopes.dtype == torch.float32
+    _check(load().opt_gqa_paged_attention_decode_no_alloc(
+        _ptr(out), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables), block_tables.shape[1],
+        _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size,
+        max_partitions, _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_decode_no_alloc")
 
 
 def paged_attention_reduce(out, partial_out, partial_lse, context_lens, partition_size: int, stream=None) -> None:

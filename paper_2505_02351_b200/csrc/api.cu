@@ -7,7 +7,7 @@ namespace optgqa {
 // Written by kernels whose bounded waits give up; read and cleared by opt_gqa_device_status().
 __device__ int g_device_status = 0;
 
-static int* device_status_ptr() {
+int* device_status_ptr() {
     static int* ptrs[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
@@ -303,6 +303,7 @@ const char* opt_gqa_status_string(int status) {
         case OPT_GQA_ERR_ALIGN: return "a data pointer is not 16-byte aligned";
         case OPT_GQA_ERR_CUDA: return "CUDA runtime error";
         case OPT_GQA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case OPT_GQA_ERR_SCRATCH: return "the call needs more scratch than the library's built-in array holds";
     }
     return "unknown status";
 }

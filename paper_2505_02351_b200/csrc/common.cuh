@@ -124,6 +124,9 @@ struct Store<__nv_bfloat16> {
     static constexpr int kDtype = OPT_GQA_BF16;
 };
 
+// Address of the current device's status word (api.cu); nullptr if the runtime refuses.
+int* device_status_ptr();
+
 // ----------------------------------------------------------------------------- host-side launchers (one per .cu)
 int launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                         const int64_t* slot_mapping, int T, int Hkv, int D, int bs, int dtype,
