@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 DEFAULT_PARTITION = {2: 256, 3: 512, 4: 512}
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised
 # under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {3: 378_700_288 + 8_656_896}   # profiles/decode_stream_cfg3.md
 
 
 # ----------------------------------------------------------------------------- distributed plumbing
@@ -308,21 +308,12 @@ def check(rc: int, what: str):
         raise RuntimeError(f"{what} failed with status {rc}")
 
 
-EVENT_EVERY = 8   # every 8th timed step brackets its decode launch with CUDA events
+EVENT_EVERY = 8   # in the kernel-timing region every 8th step carries an event bracket
+DECODE_BATCH = 4  # decode launches inside one bracket
 
 
-def run_timed(batch: DeviceBatch, steps: int, warmup: int, per_kernel_events: bool):
-    """Warm-up, then `steps` steps timed with CUDA events on the launching stream.
-
-    A step is one opt_gqa_decode_step call (append -> decode -> reduce, chained with programmatic
-    dependent launches).  Every EVENT_EVERY-th step is issued as the three separate calls instead, with
-    an event before and after the decode launch: those samples give the decode kernel's average
-    duration inside the timed region without putting event records between the kernels of every step.
-    Returns (total_ms, decode_ms_avg or None, launches).  Consecutive steps use different pool copies.
-    """
-    import torch
-
-    stream = torch.cuda.current_stream()
+def _step_fns(batch: DeviceBatch, stream):
+    """Pre-marshalled foreign calls of one step, per pool copy."""
     sh = stream.cuda_stream
     lib, R, split = batch.lib, len(batch.k_pools), batch.P > 0
     a_app = [batch.args_append(i, sh) for i in range(R)]
@@ -335,35 +326,78 @@ def run_timed(batch: DeviceBatch, steps: int, warmup: int, per_kernel_events: bo
     else:
         f_dec, f_red = lib.opt_gqa_paged_attention_decode, lib.opt_gqa_paged_attention_reduce
     f_step = lib.opt_gqa_decode_step
+    return dict(R=R, split=split, append=lambda i: check(f_app(*a_app[i % R]), "cache_append"),
+                decode=lambda i: check(f_dec(*a_dec[i % R]), "decode"),
+                reduce=lambda: check(f_red(*a_red), "reduce") if split else None,
+                step=lambda i: check(f_step(*a_step[i % R]), "decode_step"))
 
-    def step(i, ev=None):
-        if ev is None:
-            check(f_step(*a_step[i % R]), "decode_step")
-            return
-        check(f_app(*a_app[i % R]), "cache_append")
-        ev[0].record(stream)
-        check(f_dec(*a_dec[i % R]), "decode")
-        ev[1].record(stream)
-        if split:
-            check(f_red(*a_red), "reduce")
 
+def run_timed(batch: DeviceBatch, steps: int, warmup: int):
+    """Warm-up, then `steps` steps timed with CUDA events on the launching stream.
+
+    A step is one opt_gqa_decode_step call (append -> decode -> reduce, chained with programmatic dependent
+    launches); consecutive steps use different pool copies.  Returns (total_ms, launches).
+    """
+    import torch
+
+    stream = torch.cuda.current_stream()
+    f = _step_fns(batch, stream)
     for i in range(warmup):
-        step(i)
+        f["step"](i)
     torch.cuda.synchronize()
-    evs = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-           for i in range(0, steps, EVENT_EVERY)} if per_kernel_events else {}
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     torch.cuda.synchronize()
     start.record(stream)
     for i in range(steps):
-        step(warmup + i, evs.get(i))
+        f["step"](warmup + i)
     end.record(stream)
     torch.cuda.synchronize()
     barrier()
-    total_ms = start.elapsed_time(end)
-    dec_ms = sum(a.elapsed_time(b) for a, b in evs.values()) / len(evs) if evs else None
-    return total_ms, dec_ms, steps * (3 if split else 2)
+    return start.elapsed_time(end), steps * (3 if f["split"] else 2)
+
+
+def run_kernel_timing(batch: DeviceBatch, steps: int, warmup: int):
+    """A second timed region of the same steps that isolates the decode kernel's launch duration.
+
+    Every EVENT_EVERY-th step is issued as separate calls with an event bracket around its decode work.  Even
+    samples bracket DECODE_BATCH back-to-back decode launches on successive pool copies (the span divided by
+    DECODE_BATCH is the duration of one launch in a pipelined stream: the launches are chained by programmatic
+    dependent launch exactly as append -> decode is in a step, so the bracket's own event and launch gaps are
+    paid once per DECODE_BATCH launches); odd samples bracket a single launch (which also pays those gaps).
+    Returns (ms per launch from the batched brackets, ms per launch from the single brackets, launches).
+    """
+    import torch
+
+    stream = torch.cuda.current_stream()
+    f = _step_fns(batch, stream)
+    for i in range(warmup):
+        f["step"](i)
+    torch.cuda.synchronize()
+    samples = list(range(0, steps, EVENT_EVERY))
+    evs = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for i in samples}
+    launches = 0
+    barrier()
+    torch.cuda.synchronize()
+    for i in range(steps):
+        if i not in evs:
+            f["step"](warmup + i)
+            launches += 3 if f["split"] else 2
+            continue
+        nb = DECODE_BATCH if (i // EVENT_EVERY) % 2 == 0 else 1
+        f["append"](warmup + i)
+        evs[i][0].record(stream)
+        for j in range(nb):
+            f["decode"](warmup + i + j)
+        evs[i][1].record(stream)
+        f["reduce"]()
+        launches += 1 + nb + (1 if f["split"] else 0)
+    torch.cuda.synchronize()
+    barrier()
+    batched = [evs[i][0].elapsed_time(evs[i][1]) / DECODE_BATCH for i in samples if (i // EVENT_EVERY) % 2 == 0]
+    single = [evs[i][0].elapsed_time(evs[i][1]) for i in samples if (i // EVENT_EVERY) % 2 == 1]
+    mean = lambda v: sum(v) / len(v) if v else None
+    return mean(batched), mean(single), launches
 
 
 def run_e2e(batch: DeviceBatch, steps: int, warmup: int):
@@ -539,7 +573,9 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    total_ms, dec_ms, launches = run_timed(batch, steps, warmup, per_kernel_events=True)
+    total_ms, launches = run_timed(batch, steps, warmup)
+    dec_ms, dec_single_ms, launches2 = run_kernel_timing(batch, min(steps, 1024), 8)
+    launches += launches2
     clocks = sampler.stop()
     status = binding.device_status()
     if status != 0:
@@ -562,6 +598,9 @@ def main():
     roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (balanced split)" if batch.balanced else "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(args.config),
                 "algorithmic_bytes_per_launch": alg, "kernel_us": dec_ms * 1e3,
+                "kernel_us_single_launch_bracket": None if dec_single_ms is None else dec_single_ms * 1e3,
+                "timing": f"CUDA events around {DECODE_BATCH} back-to-back decode launches on successive pool copies, "
+                          f"every {2 * EVENT_EVERY}th step of a second timed region; span / {DECODE_BATCH}",
                 "frac_of_nominal_8TBs": achieved / 8000.0}
 
     line = {
@@ -589,7 +628,8 @@ def main():
                 continue
             w2 = W.make_config(cfg)
             b2 = DeviceBatch(w2, w2.partition_size or DEFAULT_PARTITION[cfg], args.copies, dev)
-            t_ms, d_ms, _ = run_timed(b2, 1000, 20, per_kernel_events=True)
+            t_ms, _ = run_timed(b2, 1000, 20)
+            d_ms, _, _ = run_kernel_timing(b2, 256, 8)
             a2 = b2.algorithmic_bytes()
             extra[w2.name] = {"tokens_per_s": w2.B * 1000 / (t_ms * 1e-3), "ms_per_step": t_ms / 1000,
                               "decode_us": d_ms * 1e3, "decode_GBs": a2 / (d_ms * 1e-3) / 1e9,
