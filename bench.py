@@ -260,7 +260,7 @@ class PrefillBatch:
         sh = stream.cuda_stream
         a_app = (self.k_new.data_ptr(), self.v_new.data_ptr(), self.k_pool.data_ptr(), self.v_pool.data_ptr(),
                  self.slots.data_ptr(), wl.T, wl.Hkv, wl.D, wl.bs, wl.num_blocks, 1, sh)
-        a_pf = (self.out.data_ptr(), self.q.data_ptr(), self.qsl.data_ptr(), self.max_q_len, self.k_pool.data_ptr(),
+        a_pf = (self.out.data_ptr(), self.q.data_ptr(), self.qsl.data_ptr(), wl.T, self.max_q_len, self.k_pool.data_ptr(),
                 self.v_pool.data_ptr(), self.tables.data_ptr(), wl.max_blocks, self.lens.data_ptr(),
                 self.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, 1, sh)
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]

@@ -204,15 +204,28 @@ int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q, const void
  * the cache; new token i sits at position pos = n_s - q_len_s + i and attends to
  * keys j <= pos with bias -slope_h*(pos - j).
  *
- *   out, q        [sum_s q_len_s, Hq, D]   (bf16 only)
+ *   out, q        [total_q_tokens, Hq, D]  (bf16 only)
  *   q_start_loc   [B+1] int32              prefix sums of q_len_s, device memory
+ *   total_q_tokens HOST value: rows of q and out (= q_start_loc[B]); rows are read up to it
  *   max_q_len     HOST value >= max_s q_len_s (sizes the grid)
+ * D = 128 runs on tcgen05.mma with accumulators in tensor memory; D = 64 on warp-level mma.
  */
-int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len,
-                                    const void* k_cache, const void* v_cache, const int32_t* block_tables,
-                                    int max_blocks_per_seq, const int32_t* context_lens,
-                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D,
-                                    int bs, int64_t num_blocks, int dtype, void* stream);
+int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+                                    int max_q_len, const void* k_cache, const void* v_cache,
+                                    const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
+                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
+                                    int64_t num_blocks, int dtype, void* stream);
+
+/*
+ * The same operation, arguments and results as opt_gqa_paged_attention_prefill, forced onto the
+ * warp-level kernel (mma.sync m16n8k16, eight consumer warps of 16 rows each and a producer warp):
+ * keeps the earlier form of Eq. 3-5 reachable for D = 128 as a cross-check and for comparison.
+ */
+int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+                                        int max_q_len, const void* k_cache, const void* v_cache,
+                                        const int32_t* block_tables, int max_blocks_per_seq,
+                                        const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                        int Hq, int Hkv, int D, int bs, int64_t num_blocks, int dtype, void* stream);
 
 /*
  * One decode step of the attention layer, Algorithm 2 from "Store reshaped K, V

@@ -35,8 +35,10 @@ SIGNATURES = {
     "opt_gqa_paged_attention_decode_no_alloc": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i,
                                                      _i64, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_reduce": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
-    "opt_gqa_paged_attention_prefill": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i,
+    "opt_gqa_paged_attention_prefill": (_i, [_vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i,
                                              _i, _i64, _i, _vp]),
+    "opt_gqa_paged_attention_prefill_mma": (_i, [_vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i,
+                                                 _i, _i, _i64, _i, _vp]),
     "opt_gqa_decode_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                  _i, _vp, _i, _i, _vp]),
     "opt_gqa_decode_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _f, _i, _i, _i, _i,
@@ -180,16 +182,28 @@ def paged_attention_reduce(out, partial_out, partial_lse, context_lens, partitio
         max_partitions, _DTYPE_CODE[out.dtype], _stream(stream)), "opt_gqa_paged_attention_reduce")
 
 
-def paged_attention_prefill(out, q, q_start_loc, max_q_len: int, k_cache, v_cache, block_tables, context_lens,
-                            alibi_slopes, scale: float, stream=None) -> None:
+def _prefill(entry: str, out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables, context_lens, alibi_slopes,
+             scale, stream) -> None:
     T, Hq, D = q.shape
     num_blocks, Hkv, bs, _ = k_cache.shape
     B = context_lens.shape[0]
     assert q_start_loc.dtype == torch.int32
-    _check(load().opt_gqa_paged_attention_prefill(
-        _ptr(out), _ptr(q), _ptr(q_start_loc), max_q_len, _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
+    _check(getattr(load(), entry)(
+        _ptr(out), _ptr(q), _ptr(q_start_loc), T, max_q_len, _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
         block_tables.shape[1], _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks,
-        _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_prefill")
+        _DTYPE_CODE[q.dtype], _stream(stream)), entry)
+
+
+def paged_attention_prefill(out, q, q_start_loc, max_q_len: int, k_cache, v_cache, block_tables, context_lens,
+                            alibi_slopes, scale: float, stream=None) -> None:
+    _prefill("opt_gqa_paged_attention_prefill", out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables,
+             context_lens, alibi_slopes, scale, stream)
+
+
+def paged_attention_prefill_mma(out, q, q_start_loc, max_q_len: int, k_cache, v_cache, block_tables, context_lens,
+                                alibi_slopes, scale: float, stream=None) -> None:
+    _prefill("opt_gqa_paged_attention_prefill_mma", out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables,
+             context_lens, alibi_slopes, scale, stream)
 
 
 def step_staging_bytes(B: int, Hq: int, Hkv: int, D: int, max_blocks_per_seq: int, dtype: torch.dtype) -> int:

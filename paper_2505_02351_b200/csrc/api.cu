@@ -160,24 +160,49 @@ int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, co
                                   static_cast<cudaStream_t>(stream));
 }
 
-int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len,
-                                    const void* k_cache, const void* v_cache, const int32_t* block_tables,
-                                    int max_blocks_per_seq, const int32_t* context_lens,
-                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
-                                    int64_t num_blocks, int dtype, void* stream) {
+static int prefill_checked(bool allow_umma, void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+                           int max_q_len, const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                           int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,
+                           float scale, int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int dtype,
+                           void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
-    if (B < 0 || max_q_len < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0)
+    if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 ||
+        num_blocks < 0)
         return OPT_GQA_ERR_SHAPE;
-    if (B == 0 || max_q_len == 0) return OPT_GQA_OK;
+    if (B == 0 || max_q_len == 0 || total_q_tokens == 0) return OPT_GQA_OK;
     if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
     if (!out || !q || !q_start_loc || !k_cache || !v_cache || !block_tables || !context_lens) return OPT_GQA_ERR_NULL;
     if (!aligned16(out) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
+    if (allow_umma && D == 128)
+        return launch_prefill_umma(out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
+                                   max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, bs, num_blocks,
+                                   status, static_cast<cudaStream_t>(stream));
     return launch_prefill(out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables, max_blocks_per_seq,
                           context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, status,
                           static_cast<cudaStream_t>(stream));
+}
+
+int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+                                    int max_q_len, const void* k_cache, const void* v_cache,
+                                    const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
+                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
+                                    int64_t num_blocks, int dtype, void* stream) {
+    return prefill_checked(true, out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
+                           max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, dtype,
+                           stream);
+}
+
+int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+                                        int max_q_len, const void* k_cache, const void* v_cache,
+                                        const int32_t* block_tables, int max_blocks_per_seq,
+                                        const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                        int Hq, int Hkv, int D, int bs, int64_t num_blocks, int dtype, void* stream) {
+    return prefill_checked(false, out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
+                           max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, dtype,
+                           stream);
 }
 
 int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,

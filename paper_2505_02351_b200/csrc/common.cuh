@@ -187,4 +187,10 @@ int launch_prefill(void* out, const void* q, const int32_t* q_start_loc, int max
                    const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
                    int D, int bs, int64_t num_blocks, int* device_status, cudaStream_t stream);
 
+// bf16, D = 128: tcgen05.mma with accumulators in tensor memory (prefill_umma.cu).
+int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens, int max_q_len,
+                        const void* k_cache, const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
+                        const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
+                        int bs, int64_t num_blocks, int* device_status, cudaStream_t stream);
+
 }  // namespace optgqa

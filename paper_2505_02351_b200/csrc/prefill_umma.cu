@@ -1,0 +1,539 @@
+// Multi-token (chunked-prefill) GQA-ALiBi attention over the paged cache on the 5th-generation
+// tensor cores: tcgen05.mma with accumulators in tensor memory (the prompt branch of Algorithms 1
+// and 2 with "Create ALiBi bias" and the causal mask; Eq. 3-5).  bf16, head_dim 128.
+//
+// One CTA per (query block, KV head, sequence).  The G query heads of the group times TQ = 128 / G
+// consecutive new tokens are the 128 rows of the CTA's tiles, so every K/V tile is fetched once for
+// the whole group ("Shared Key-Value").  Six warps, three roles:
+//   warps 0-3  one thread per row: read a 128 x 128 score tile S from tensor memory, add the ALiBi
+//              term slope_h*(j - pos) and mask j > pos from the indices (Eq. 3), keep the row's
+//              running maximum and denominator (Eq. 4, online), write p as bf16 back into tensor
+//              memory over S, rescale O when the maximum moved, and store the normalised rows
+//   warp 4     producer: walks the block table and fetches 128-key K and V tiles (2-D TMA boxes of
+//              16 token rows x 128 bytes, 128-byte swizzle) into a three-stage ring, plus the Q tile
+//   warp 5     one thread issues S = Q K^T (operands in shared memory) and O += P V (P from tensor
+//              memory, V in shared memory addressed MN-major) and commits them to mbarriers
+// S is double-buffered in tensor memory, so the tensor core works on tile j+1's scores and tile
+// j-1's P V while the row threads do tile j's softmax.  Every wait is a bounded mbarrier wait.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace optgqa {
+
+namespace {
+
+constexpr int kD = 128;            // head dimension
+constexpr int kRows = 128;         // rows of the CTA's tiles (G heads x TQ tokens)
+constexpr int kTN = 128;           // keys per tile
+constexpr int kSub = 16;           // token rows per TMA box
+constexpr int kKvStages = 3;
+constexpr int kThreads = 192;
+constexpr unsigned kFull = 0xffffffffu;
+constexpr float kRescaleThreshold = 8.f;   // log2 units: O is rescaled only when a row's maximum grew by more
+
+constexpr int kHalfBytes = kTN * 128;              // one 64-dim column half of a 128-row tile: 16 KiB
+constexpr int kTileBytes = 2 * kHalfBytes;         // a Q, K or V tile: 32 KiB
+constexpr int kOffQ = 0;
+constexpr int kOffK = kTileBytes;
+constexpr int kOffV = kOffK + kKvStages * kTileBytes;
+constexpr int kOffBar = kOffV + kKvStages * kTileBytes;
+// barriers: q_full, k_full[3], k_empty[3], v_full[3], v_empty[3], s_full[2], p_full[2]; then the TMEM base word
+constexpr int kNumBars = 1 + 4 * kKvStages + 4;
+constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;   // + slack to align the tiles to 1 KiB
+
+// tensor-memory columns (fp32 accumulators, 128 lanes each)
+constexpr uint32_t kColS = 0;       // S buffers at 0 and 128; P (bf16 pairs) overlays the first 64 columns of its S
+constexpr uint32_t kColO = 256;
+constexpr uint32_t kTmemCols = 512;
+
+struct UmmaParams {
+    __nv_bfloat16* out;
+    const int32_t* q_start_loc;
+    const int32_t* block_tables;
+    const int32_t* context_lens;
+    const float* slopes;
+    int* status;
+    float scale;
+    int max_blocks;
+    int Hq;
+    int Hkv;
+    int bs;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Arrives on `bar` once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+// Shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = N = 128, A K-major, B K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+          "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+          "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_v, const UmmaParams p) {
+    constexpr int TQ = kRows / G;     // new tokens per query block
+    extern __shared__ char smem_raw[];
+    char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kOffBar);
+    uint64_t* q_full = bars;
+    uint64_t* k_full = bars + 1;
+    uint64_t* k_empty = k_full + kKvStages;
+    uint64_t* v_full = k_empty + kKvStages;
+    uint64_t* v_empty = v_full + kKvStages;
+    uint64_t* s_full = v_empty + kKvStages;
+    uint64_t* p_full = s_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
+
+    grid_dependency_launch();
+    const int kvh = blockIdx.y, s = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qstart = p.q_start_loc[s];
+    const int qlen = p.q_start_loc[s + 1] - qstart;
+    const int nblk = (qlen + TQ - 1) / TQ;
+    if ((int)blockIdx.x >= nblk) return;
+    const int qb = nblk - 1 - (int)blockIdx.x;             // the longest-running blocks start first
+    const int n = p.context_lens[s];
+    const int i_last = min(qlen, (qb + 1) * TQ) - 1;        // last valid new token of this block
+    const int pos_last = n - qlen + i_last;                 // its position; the block sees keys 0 .. pos_last
+    const int ntiles = pos_last / kTN + 1;
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+#pragma unroll
+        for (int i = 0; i < kKvStages; ++i) {
+            mbar_init(&k_full[i], 1);
+            mbar_init(&k_empty[i], 1);
+            mbar_init(&v_full[i], 1);
+            mbar_init(&v_empty[i], 1);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_full[i], kRows);
+        }
+        tmem_slot[1] = 0;       // set by mbar_wait's callers when a wait gave up (see the end of the kernel)
+        fence_barrier_init();
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    grid_dependency_wait();     // the cache may still be receiving this step's appended tokens
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            mbar_expect_tx(q_full, kTileBytes);
+            tma_load_3d(smem + kOffQ, &map_q, 0, kvh * G, qstart + qb * TQ, q_full);
+            tma_load_3d(smem + kOffQ + kHalfBytes, &map_q, 64, kvh * G, qstart + qb * TQ, q_full);
+        }
+        const int32_t* table = p.block_tables + (size_t)s * p.max_blocks;
+        const int sub = lane & 7;                           // lanes 0-7 fetch one 16-token slice each
+        auto page_of = [&](int j) -> int {
+            const int tok = j * kTN + sub * kSub;
+            return (lane < 8 && tok < n) ? __ldg(table + tok / p.bs) : -1;
+        };
+        int page = page_of(0);
+        for (int j = 0; j < ntiles; ++j) {
+            const int st = j % kKvStages;
+            const int page_next = j + 1 < ntiles ? page_of(j + 1) : -1;
+            const int j0 = j * kTN;
+            const int nsub = min(kTN / kSub, (n - j0 + kSub - 1) / kSub);     // slices that hold cached tokens
+            const int tok = j0 + sub * kSub;
+            const int row = (page * p.Hkv + kvh) * p.bs + tok % p.bs;          // row of the [rows, D] view
+            bool ok = true;
+            if (j >= kKvStages) ok = mbar_wait(&k_empty[st], ((j / kKvStages) - 1) & 1, p.status);
+            if (!__all_sync(kFull, ok)) break;
+            if (lane == 0) mbar_expect_tx(&k_full[st], (uint32_t)nsub * 2u * kSub * 128u);
+            __syncwarp();
+            if (lane < nsub) {
+                char* dst = smem + kOffK + st * kTileBytes + sub * (kSub * 128);
+                tma_load_2d(dst, &map_k, 0, row, &k_full[st]);
+                tma_load_2d(dst + kHalfBytes, &map_k, 64, row, &k_full[st]);
+            }
+            if (j >= kKvStages) ok = mbar_wait(&v_empty[st], ((j / kKvStages) - 1) & 1, p.status);
+            if (!__all_sync(kFull, ok)) break;
+            if (lane == 0) mbar_expect_tx(&v_full[st], (uint32_t)nsub * 2u * kSub * 128u);
+            __syncwarp();
+            if (lane < nsub) {
+                char* dst = smem + kOffV + st * kTileBytes + sub * (kSub * 128);
+                tma_load_2d(dst, &map_v, 0, row, &v_full[st]);
+                tma_load_2d(dst + kHalfBytes, &map_v, 64, row, &v_full[st]);
+            }
+            page = page_next;
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ tensor-core issue (one thread)
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(false), idesc_pv = instr_desc(true);
+            const uint32_t q_addr = smem_u32(smem + kOffQ);
+            bool ok = mbar_wait(q_full, 0, p.status);
+            // O += P V for tile t: P (bf16 pairs, 8 columns per 16 keys) from tensor memory, V addressed MN-major:
+            // 64-dim halves kHalfBytes apart (leading offset), groups of 8 keys 1 KiB apart (stride offset).
+            auto issue_pv = [&](int t) -> bool {
+                const int st = t % kKvStages, sb = t & 1;
+                if (!mbar_wait(&p_full[sb], (t >> 1) & 1, p.status)) return false;
+                if (!mbar_wait(&v_full[st], (t / kKvStages) & 1, p.status)) return false;
+                tc_fence_after();
+                const uint32_t v_addr = smem_u32(smem + kOffV + st * kTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < kTN / 16; ++kk)
+                    umma_ts(tmem_base + kColO, tmem_base + kColS + sb * 128 + kk * 8,
+                            smem_desc(v_addr + kk * 2048, kHalfBytes, 1024), idesc_pv, t > 0 || kk > 0);
+                tc_commit(&v_empty[st]);
+                return true;
+            };
+            for (int j = 0; ok && j < ntiles; ++j) {
+                const int st = j % kKvStages, sb = j & 1;
+                ok = mbar_wait(&k_full[st], (j / kKvStages) & 1, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                // S = Q K^T: both K-major, 16 dims (32 bytes) per step inside the 128-byte swizzled rows
+                const uint32_t k_addr = smem_u32(smem + kOffK + st * kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < kD / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                    umma_ss(tmem_base + kColS + sb * 128, smem_desc(q_addr + off, 16, 1024),
+                            smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                }
+                tc_commit(&s_full[sb]);
+                tc_commit(&k_empty[st]);
+                if (j >= 1) ok = issue_pv(j - 1);
+            }
+            if (ok) issue_pv(ntiles - 1);
+        }
+    } else {
+        // ------------------------------------------------------------------ one thread per row: softmax, rescale, store
+        const int r = threadIdx.x;                    // row of the tiles = tensor-memory lane
+        const int tok = r / G, hg = r % G;            // the Q box is filled head-fastest
+        const int i = qb * TQ + tok;                  // new-token index in the sequence
+        const bool valid = i < qlen;
+        // Rows past the end of the block are computed as copies of the last valid position and never stored.
+        const int pos = n - qlen + min(i, i_last);
+        const int h = kvh * G + hg;
+        const float qscale = p.scale * kLog2e;
+        const float slope2 = p.slopes ? p.slopes[h] * kLog2e : 0.f;
+        const float c_row = -slope2 * (float)pos;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        float m_used = -INFINITY, l = 0.f;
+        bool ok = true;
+
+        for (int j = 0; j < ntiles; ++j) {
+            const int sb = j & 1, j0 = j * kTN;
+            ok = __all_sync(kFull, mbar_wait(&s_full[sb], (j >> 1) & 1, p.status));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t s_addr = lane_addr + kColS + sb * 128;
+
+            // ---- scores of the row for the tile's 128 keys (Eq. 3), their maximum
+            float sc[kTN];
+            float m_tile = -INFINITY;
+            const bool masked = j0 + kTN - 1 > pos;
+#pragma unroll
+            for (int c = 0; c < kTN / 32; ++c) {
+                float v[32];
+                tmem_ld32(s_addr + c * 32, v);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int jj = j0 + c * 32 + e;
+                    float t = fmaf(v[e], qscale, fmaf(slope2, (float)jj, c_row));
+                    if (masked) t = jj <= pos ? t : -INFINITY;
+                    sc[c * 32 + e] = t;
+                    m_tile = fmaxf(m_tile, t);
+                }
+            }
+
+            // ---- running maximum: move it (and rescale l and O) only when it grew by more than the threshold
+            const bool need = m_tile > m_used + kRescaleThreshold;     // true on the first tile (m_used = -inf)
+            const float m_new = need ? m_tile : m_used;
+            const float f = need ? ex2(m_used - m_new) : 1.f;          // 0 on the first tile
+            if (j > 0 && __any_sync(kFull, need)) {
+                // O holds tiles 0 .. j-1 once tile j-1's P V has completed
+                ok = __all_sync(kFull, mbar_wait(&v_empty[(j - 1) % kKvStages], ((j - 1) / kKvStages) & 1, p.status));
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < kD / 32; ++c) {
+                    float v[32];
+                    uint32_t w[32];
+                    tmem_ld32(lane_addr + kColO + c * 32, v);
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) w[e] = __float_as_uint(v[e] * f);
+                    tmem_st32(lane_addr + kColO + c * 32, w);
+                }
+            }
+            m_used = m_new;
+            l *= f;
+
+            // ---- p = 2^(s - m) (Eq. 4), rounded to bf16 pairs over the first 64 columns of S
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t w[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float p0 = ex2(sc[c * 64 + 2 * e] - m_used), p1 = ex2(sc[c * 64 + 2 * e + 1] - m_used);
+                    sum += p0 + p1;
+                    w[e] = pack2(p0, p1);
+                }
+                tmem_st32(s_addr + c * 32, w);
+            }
+            l += sum;
+
+            if (j0 + kTN > n) {
+                // Rows past the end of the sequence hold whatever the page held, or stale shared memory where no
+                // page exists: zero this thread's V row so that 0 * garbage cannot produce NaN.
+                const int st = j % kKvStages;
+                ok = __all_sync(kFull, mbar_wait(&v_full[st], (j / kKvStages) & 1, p.status));
+                if (!ok) break;
+                if (j0 + r >= n) {
+                    char* vrow = smem + kOffV + st * kTileBytes + r * 128;
+#pragma unroll
+                    for (int b = 0; b < 2; ++b)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            *reinterpret_cast<uint4*>(vrow + b * kHalfBytes + e * 16) = make_uint4(0, 0, 0, 0);
+                    fence_proxy_async();
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&p_full[sb]);
+        }
+
+        if (ok) {
+            // ---- all tiles accumulated once the last P V has completed: normalise (Eq. 5) and store
+            ok = __all_sync(kFull, mbar_wait(&v_empty[(ntiles - 1) % kKvStages], ((ntiles - 1) / kKvStages) & 1, p.status));
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.f / l;
+            uint4* orow = reinterpret_cast<uint4*>(p.out + ((size_t)(qstart + i) * p.Hq + h) * kD);
+#pragma unroll
+            for (int c = 0; c < kD / 32; ++c) {
+                float v[32];
+                tmem_ld32(lane_addr + kColO + c * 32, v);
+                if (valid) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        orow[c * 4 + e] = make_uint4(pack2(v[8 * e] * inv, v[8 * e + 1] * inv),
+                                                     pack2(v[8 * e + 2] * inv, v[8 * e + 3] * inv),
+                                                     pack2(v[8 * e + 4] * inv, v[8 * e + 5] * inv),
+                                                     pack2(v[8 * e + 6] * inv, v[8 * e + 7] * inv));
+                }
+            }
+        }
+    }
+
+    // ---- every role is done with tensor memory: give it back.  If a bounded wait gave up somewhere (already
+    // recorded in the status word), copies or tensor-core work of this CTA may still be in flight: let them
+    // drain for a while before the shared and tensor memory are released.
+    if (*reinterpret_cast<volatile int*>(p.status) != 0) tmem_slot[1] = 1;
+    tc_fence_before();
+    __syncthreads();
+    if (tmem_slot[1]) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// The cache seen as a 2-D bf16 tensor [num_blocks*Hkv*bs rows, 128]; a box is 16 token rows x 64 dims (128 B).
+bool make_cache_map(CUtensorMap* map, const void* cache, uint64_t rows) {
+    EncodeFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kSub};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// q [tokens, Hq, 128] as a 3-D tensor; a box is 64 dims x the G heads of a group x 128 / G tokens, i.e. one
+// 64-dim half of the CTA's 128 rows, head-fastest.  Tokens past the end of q read as zeros.
+bool make_q_map(CUtensorMap* map, const void* q, int tokens, int Hq, int G) {
+    EncodeFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hq, (cuuint64_t)tokens};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hq * kD * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(kRows / G)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int G>
+int launch_one(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& p, int B,
+               int max_q_len, cudaStream_t stream) {
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    if (dev < 64 && !configured[dev]) {
+        if (cudaFuncSetAttribute(prefill_umma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+            cudaSuccess)
+            return OPT_GQA_ERR_CUDA;
+        configured[dev] = true;
+    }
+    constexpr int TQ = kRows / G;
+    dim3 grid((max_q_len + TQ - 1) / TQ, p.Hkv, B);
+    return launch_dependent(prefill_umma_kernel<G>, grid, dim3(kThreads), kSmemBytes, stream, mq, mk, mv, p);
+}
+
+}  // namespace
+
+// bf16, D = 128 only.
+int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens, int max_q_len,
+                        const void* k_cache, const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
+                        const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
+                        int bs, int64_t num_blocks, int* device_status, cudaStream_t stream) {
+    const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
+    if (rows == 0 || rows > 0x7fffffffull || total_q_tokens <= 0) return OPT_GQA_ERR_SHAPE;
+    if (B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
+    const int G = Hq / Hkv;
+    CUtensorMap mq, mk, mv;
+    if (!make_q_map(&mq, q, total_q_tokens, Hq, G) || !make_cache_map(&mk, k_cache, rows) ||
+        !make_cache_map(&mv, v_cache, rows))
+        return OPT_GQA_ERR_CUDA;
+    UmmaParams p;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.q_start_loc = q_start_loc;
+    p.block_tables = block_tables;
+    p.context_lens = context_lens;
+    p.slopes = alibi_slopes;
+    p.status = device_status;
+    p.scale = scale;
+    p.max_blocks = max_blocks_per_seq;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.bs = bs;
+    switch (G) {
+        case 1: return launch_one<1>(mq, mk, mv, p, B, max_q_len, stream);
+        case 2: return launch_one<2>(mq, mk, mv, p, B, max_q_len, stream);
+        case 4: return launch_one<4>(mq, mk, mv, p, B, max_q_len, stream);
+        case 8: return launch_one<8>(mq, mk, mv, p, B, max_q_len, stream);
+    }
+    return OPT_GQA_ERR_SHAPE;
+}
+
+}  // namespace optgqa

@@ -30,6 +30,27 @@ def test_shape_matrix_ragged_chunks(D, Hq, Hkv, bs):
     wl = W.make_custom("pf", "bf16", Hq, Hkv, D, bs, lens, q_lens=qls, seed=D + Hq + bs, poison=True)
     _check(wl)
     _check(wl, slopes=False)
+    if D == 128:                 # the default entry point ran on tcgen05: also the warp-level kernel
+        _check(wl, mma=True)
+
+
+def test_tiles_and_blocks_boundaries_on_tcgen05():
+    # contexts and chunks around the 128-key tile and the 128-row query block: exactly full, one over, one under
+    for G, Hkv in ((4, 2), (8, 1), (1, 2), (2, 2)):
+        TQ = 128 // G
+        lens = [128, 129, 127, 256 + TQ, 3 * 128 + 1, 640, 5]
+        qls = [min(a, b) for a, b in zip(lens, [128, 1, TQ, TQ + 1, 2 * TQ - 1, 640, 5])]
+        wl = W.make_custom("edge", "bf16", G * Hkv, Hkv, 128, 16, lens, q_lens=qls, seed=50 + G, poison=True)
+        _check(wl)
+
+
+def test_large_maximum_drift_forces_rescales():
+    # scores that keep growing along the context (steep negative ALiBi slope is the usual case; here the values of
+    # q.k themselves grow), so the running maximum moves by more than the rescale threshold many times
+    wl = W.make_custom("drift", "bf16", 4, 1, 128, 16, [1500], q_lens=[300], seed=51,
+                       slopes=torch.tensor([4.0, 1.0, 0.25, 0.0]), scale=1.0)
+    _check(wl)
+    _check(wl, mma=True)
 
 
 def test_config5_shrunk():
@@ -37,6 +58,7 @@ def test_config5_shrunk():
     wl = W.make_config(5, shrink=8, poison=True)
     assert wl.T == 4 * 256
     _check(wl)
+    _check(wl, mma=True)
 
 
 def test_prefill_with_one_new_token_is_the_decode_result():

@@ -69,21 +69,24 @@ def oracle_inputs(wl: W.Workload, append=True):
                 qsl=None if wl.q_start_loc is None else wl.q_start_loc.numpy())
 
 
-def oracle_attention(wl: W.Workload, append=True, slopes=True, simt=False, balanced=False):
+def oracle_attention(wl: W.Workload, append=True, slopes=True, simt=False, balanced=False, mma=False):
     a = oracle_inputs(wl, append)
     return oracle.paged_attention(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"] if slopes else None, wl.scale,
                                   wl.dtype, q_start_loc=a["qsl"])
 
 
-def gpu_prefill(wl: W.Workload, append=True, slopes=True):
-    """append + chunked prefill through the C ABI; returns (out float64 numpy, DeviceWorkload)."""
+def gpu_prefill(wl: W.Workload, append=True, slopes=True, mma=False):
+    """append + chunked prefill through the C ABI; returns (out float64 numpy, DeviceWorkload).
+
+    mma=True forces the warp-level kernel (the default entry point runs D = 128 on tcgen05)."""
     d = DeviceWorkload(wl)
     if append:
         binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
     qsl = wl.q_start_loc.numpy()
     max_q_len = int((qsl[1:] - qsl[:-1]).max()) if wl.B else 0
-    binding.paged_attention_prefill(d.out, d.q, d.q_start_loc, max_q_len, d.k_cache, d.v_cache, d.block_tables,
-                                    d.context_lens, d.alibi_slopes if slopes else None, wl.scale)
+    fn = binding.paged_attention_prefill_mma if mma else binding.paged_attention_prefill
+    fn(d.out, d.q, d.q_start_loc, max_q_len, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+       d.alibi_slopes if slopes else None, wl.scale)
     torch.cuda.synchronize()
     assert binding.device_status() == 0
     return d.out.double().cpu().numpy(), d
