@@ -14,7 +14,10 @@
 //   warp 5     one thread issues S = Q K^T (operands in shared memory) and O += P V (P from tensor
 //              memory, V in shared memory addressed MN-major) and commits them to mbarriers
 // S is double-buffered in tensor memory, so the tensor core works on tile j+1's scores and tile
-// j-1's P V while the row threads do tile j's softmax.  Every wait is a bounded mbarrier wait.
+// j-1's P V while the row threads do tile j's softmax.  Tiles are taken from the diagonal backwards
+// (nearest keys first): the ALiBi term falls with distance, so a row's maximum is set by the first
+// tiles it sees and O is rescaled only when the maximum still grows by more than 2^8 -- in forward
+// order the bias alone would move it every tile.  Every wait is a bounded mbarrier wait.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -227,15 +230,15 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         const int32_t* table = p.block_tables + (size_t)s * p.max_blocks;
         const int sub = lane & 7;                           // lanes 0-7 fetch one 16-token slice each
-        auto page_of = [&](int j) -> int {
-            const int tok = j * kTN + sub * kSub;
+        auto page_of = [&](int j) -> int {         // j counts processed tiles; the tile is ntiles - 1 - j
+            const int tok = (ntiles - 1 - j) * kTN + sub * kSub;
             return (lane < 8 && tok < n) ? __ldg(table + tok / p.bs) : -1;
         };
         int page = page_of(0);
         for (int j = 0; j < ntiles; ++j) {
             const int st = j % kKvStages;
             const int page_next = j + 1 < ntiles ? page_of(j + 1) : -1;
-            const int j0 = j * kTN;
+            const int j0 = (ntiles - 1 - j) * kTN;
             const int nsub = min(kTN / kSub, (n - j0 + kSub - 1) / kSub);     // slices that hold cached tokens
             const int tok = j0 + sub * kSub;
             const int row = (page * p.Hkv + kvh) * p.bs + tok % p.bs;          // row of the [rows, D] view
@@ -317,7 +320,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         bool ok = true;
 
         for (int j = 0; j < ntiles; ++j) {
-            const int sb = j & 1, j0 = j * kTN;
+            const int sb = j & 1, j0 = (ntiles - 1 - j) * kTN;
             ok = __all_sync(kFull, mbar_wait(&s_full[sb], (j >> 1) & 1, p.status));
             if (!ok) break;
             tc_fence_after();
@@ -327,6 +330,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             float sc[kTN];
             float m_tile = -INFINITY;
             const bool masked = j0 + kTN - 1 > pos;
+            const float bias0 = fmaf(slope2, (float)j0, c_row);       // ALiBi term of the tile's first key
 #pragma unroll
             for (int c = 0; c < kTN / 32; ++c) {
                 float v[32];
@@ -334,7 +338,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     const int jj = j0 + c * 32 + e;
-                    float t = fmaf(v[e], qscale, fmaf(slope2, (float)jj, c_row));
+                    float t = fmaf(v[e], qscale, fmaf(slope2, (float)(c * 32 + e), bias0));
                     if (masked) t = jj <= pos ? t : -INFINITY;
                     sc[c * 32 + e] = t;
                     m_tile = fmaxf(m_tile, t);
@@ -342,9 +346,10 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             }
 
             // ---- running maximum: move it (and rescale l and O) only when it grew by more than the threshold
-            const bool need = m_tile > m_used + kRescaleThreshold;     // true on the first tile (m_used = -inf)
+            // (true for the first tile in which the row sees a key: m_used = -inf until then)
+            const bool need = m_tile > m_used + kRescaleThreshold;
             const float m_new = need ? m_tile : m_used;
-            const float f = need ? ex2(m_used - m_new) : 1.f;          // 0 on the first tile
+            const float f = need ? ex2(m_used - m_new) : 1.f;          // 0 the first time
             if (j > 0 && __any_sync(kFull, need)) {
                 // O holds tiles 0 .. j-1 once tile j-1's P V has completed
                 ok = __all_sync(kFull, mbar_wait(&v_empty[(j - 1) % kKvStages], ((j - 1) / kKvStages) & 1, p.status));
@@ -364,13 +369,15 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             l *= f;
 
             // ---- p = 2^(s - m) (Eq. 4), rounded to bf16 pairs over the first 64 columns of S
+            // (a row that has not seen a key yet has only -inf scores: subtract 0 so that they give p = 0)
+            const float m_sub = m_used == -INFINITY ? 0.f : m_used;
             float sum = 0.f;
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t w[32];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    const float p0 = ex2(sc[c * 64 + 2 * e] - m_used), p1 = ex2(sc[c * 64 + 2 * e + 1] - m_used);
+                    const float p0 = ex2(sc[c * 64 + 2 * e] - m_sub), p1 = ex2(sc[c * 64 + 2 * e + 1] - m_sub);
                     sum += p0 + p1;
                     w[e] = pack2(p0, p1);
                 }
