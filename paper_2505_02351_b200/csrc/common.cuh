@@ -49,11 +49,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return done != 0;
 }
 
-// Bounded wait: gives up after kSpinLimit polls, records the timeout and returns false.
-constexpr uint32_t kSpinLimit = 1u << 22;
+// Bounded wait: gives up after about kWaitLimitCycles SM clocks (~0.14 s; real waits last microseconds), records
+// the timeout and returns false.  The bound is on elapsed time, not on the number of polls: one try_wait may
+// itself block for a while before it reports failure.
+constexpr long long kWaitLimitCycles = 1ll << 28;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    do {
         if (mbar_try_wait(bar, parity)) return true;
+    } while (clock64() - start < kWaitLimitCycles);
     atomicExch(status, OPT_GQA_ERR_TIMEOUT);
     return false;
 }

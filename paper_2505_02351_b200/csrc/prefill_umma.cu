@@ -5,19 +5,24 @@
 // One CTA per (query block, KV head, sequence).  The G query heads of the group times TQ = 128 / G
 // consecutive new tokens are the 128 rows of the CTA's tiles, so every K/V tile is fetched once for
 // the whole group ("Shared Key-Value").  Six warps, three roles:
-//   warps 0-3  one thread per row: read a 128 x 128 score tile S from tensor memory, add the ALiBi
+//   warps 0-3  one thread per row: read the 128 x kTN score tile S from tensor memory, add the ALiBi
 //              term slope_h*(j - pos) and mask j > pos from the indices (Eq. 3), keep the row's
-//              running maximum and denominator (Eq. 4, online), write p as bf16 back into tensor
-//              memory over S, rescale O when the maximum moved, and store the normalised rows
-//   warp 4     producer: walks the block table and fetches 128-key K and V tiles (2-D TMA boxes of
-//              16 token rows x 128 bytes, 128-byte swizzle) into a three-stage ring, plus the Q tile
+//              running maximum and denominator (Eq. 4, online; two passes over S, first the maximum,
+//              then p), write p as bf16 back into tensor memory over S, rescale O when the maximum
+//              moved, and store the normalised rows
+//   warp 4     producer: walks the block table and fetches kTN-key K and V tiles (2-D TMA boxes of
+//              16 token rows x 128 bytes, 128-byte swizzle) into a ring, plus the Q tile
 //   warp 5     one thread issues S = Q K^T (operands in shared memory) and O += P V (P from tensor
 //              memory, V in shared memory addressed MN-major) and commits them to mbarriers
 // S is double-buffered in tensor memory, so the tensor core works on tile j+1's scores and tile
 // j-1's P V while the row threads do tile j's softmax.  Tiles are taken from the diagonal backwards
 // (nearest keys first): the ALiBi term falls with distance, so a row's maximum is set by the first
 // tiles it sees and O is rescaled only when the maximum still grows by more than 2^8 -- in forward
-// order the bias alone would move it every tile.  Every wait is a bounded mbarrier wait.
+// order the bias alone would move it every tile.  The softmax is bound by instruction issue (exp2 on
+// the special-function unit, max on the half-rate pipe) with one row warp per scheduler, so the
+// default shape is 64-key tiles in a two-stage ring: two CTAs fit on an SM (96 KiB of shared memory
+// and 256 tensor-memory columns each) and one CTA's exp2 phase overlaps the other's maximum phase.
+// Every wait is a bounded mbarrier wait.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -28,17 +33,29 @@ namespace {
 
 constexpr int kD = 128;            // head dimension
 constexpr int kRows = 128;         // rows of the CTA's tiles (G heads x TQ tokens)
-constexpr int kTN = 128;           // keys per tile
+#ifndef OPT_GQA_PF_TN
+#define OPT_GQA_PF_TN 64
+#endif
+#ifndef OPT_GQA_PF_STAGES
+#define OPT_GQA_PF_STAGES 2
+#endif
+#ifndef OPT_GQA_PF_CTAS
+#define OPT_GQA_PF_CTAS 2
+#endif
+constexpr int kTN = OPT_GQA_PF_TN;  // keys per tile (64 or 128)
 constexpr int kSub = 16;           // token rows per TMA box
-constexpr int kKvStages = 3;
+constexpr int kKvStages = OPT_GQA_PF_STAGES;
+constexpr int kCtasPerSm = OPT_GQA_PF_CTAS;
 constexpr int kThreads = 192;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: O is rescaled only when a row's maximum grew by more
 
-constexpr int kHalfBytes = kTN * 128;              // one 64-dim column half of a 128-row tile: 16 KiB
-constexpr int kTileBytes = 2 * kHalfBytes;         // a Q, K or V tile: 32 KiB
+constexpr int kHalfBytes = kTN * 128;              // one 64-dim column half of a K or V tile (kTN rows of 128 B)
+constexpr int kTileBytes = 2 * kHalfBytes;         // a K or V tile
+constexpr int kQHalfBytes = kRows * 128;           // one 64-dim column half of the Q tile: 16 KiB
+constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kOffQ = 0;
-constexpr int kOffK = kTileBytes;
+constexpr int kOffK = kQBytes;
 constexpr int kOffV = kOffK + kKvStages * kTileBytes;
 constexpr int kOffBar = kOffV + kKvStages * kTileBytes;
 // barriers: q_full, k_full[3], k_empty[3], v_full[3], v_empty[3], s_full[2], p_full[2]; then the TMEM base word
@@ -46,9 +63,10 @@ constexpr int kNumBars = 1 + 4 * kKvStages + 4;
 constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;   // + slack to align the tiles to 1 KiB
 
 // tensor-memory columns (fp32 accumulators, 128 lanes each)
-constexpr uint32_t kColS = 0;       // S buffers at 0 and 128; P (bf16 pairs) overlays the first 64 columns of its S
-constexpr uint32_t kColO = 256;
-constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0;       // S buffers at 0 and kTN; P (bf16 pairs) overlays the first kTN / 2 columns of its S
+constexpr uint32_t kColO = 2 * kTN;
+constexpr uint32_t kTmemCols = kTN == 128 ? 512 : 256;    // a power of two >= 2 kTN + 128
+static_assert(kTN == 64 || kTN == 128, "tile of 64 or 128 keys");
 
 struct UmmaParams {
     __nv_bfloat16* out;
@@ -100,9 +118,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
            (1ull << 46) | (2ull << 61);
 }
 
-// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = N = 128, A K-major, B K-major or MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128, N = n, A K-major, B K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major, uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // D[tmem] (+)= A[smem] * B[smem]
@@ -125,9 +143,9 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
         : "memory");
 }
 
-// 32 consecutive fp32 columns of this thread's lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
+// Starts the load of 32 consecutive 32-bit columns of this thread's lane; the registers are valid only after
+// tmem_wait_ld() (and tmem_pin(), which keeps the compiler from moving their uses above the wait).
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -138,7 +156,26 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_pin(uint32_t* r) {     // 32 registers, no instruction
+#pragma unroll
+    for (int i = 0; i < 32; i += 16)
+        asm volatile("" : "+r"(r[i]), "+r"(r[i + 1]), "+r"(r[i + 2]), "+r"(r[i + 3]), "+r"(r[i + 4]), "+r"(r[i + 5]),
+                          "+r"(r[i + 6]), "+r"(r[i + 7]), "+r"(r[i + 8]), "+r"(r[i + 9]), "+r"(r[i + 10]), "+r"(r[i + 11]),
+                          "+r"(r[i + 12]), "+r"(r[i + 13]), "+r"(r[i + 14]), "+r"(r[i + 15])
+                     :
+                     : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    tmem_ld32_issue(taddr, r);
+    tmem_wait_ld();
+    tmem_pin(r);
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
@@ -155,6 +192,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr)
+        : "memory");
+}
+
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
@@ -163,7 +209,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 }
 
 template <int G>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const UmmaParams p) {
     constexpr int TQ = kRows / G;     // new tokens per query block
@@ -224,9 +270,9 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (warp == 4) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            mbar_expect_tx(q_full, kTileBytes);
+            mbar_expect_tx(q_full, kQBytes);
             tma_load_3d(smem + kOffQ, &map_q, 0, kvh * G, qstart + qb * TQ, q_full);
-            tma_load_3d(smem + kOffQ + kHalfBytes, &map_q, 64, kvh * G, qstart + qb * TQ, q_full);
+            tma_load_3d(smem + kOffQ + kQHalfBytes, &map_q, 64, kvh * G, qstart + qb * TQ, q_full);
         }
         const int32_t* table = p.block_tables + (size_t)s * p.max_blocks;
         const int sub = lane & 7;                           // lanes 0-7 fetch one 16-token slice each
@@ -266,7 +312,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     } else if (warp == 5) {
         // ------------------------------------------------------------------ tensor-core issue (one thread)
         if (lane == 0) {
-            constexpr uint32_t idesc_s = instr_desc(false), idesc_pv = instr_desc(true);
+            constexpr uint32_t idesc_s = instr_desc(false, kTN), idesc_pv = instr_desc(true, kD);
             const uint32_t q_addr = smem_u32(smem + kOffQ);
             bool ok = mbar_wait(q_full, 0, p.status);
             // O += P V for tile t: P (bf16 pairs, 8 columns per 16 keys) from tensor memory, V addressed MN-major:
@@ -279,7 +325,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 const uint32_t v_addr = smem_u32(smem + kOffV + st * kTileBytes);
 #pragma unroll
                 for (int kk = 0; kk < kTN / 16; ++kk)
-                    umma_ts(tmem_base + kColO, tmem_base + kColS + sb * 128 + kk * 8,
+                    umma_ts(tmem_base + kColO, tmem_base + kColS + sb * kTN + kk * 8,
                             smem_desc(v_addr + kk * 2048, kHalfBytes, 1024), idesc_pv, t > 0 || kk > 0);
                 tc_commit(&v_empty[st]);
                 return true;
@@ -293,9 +339,9 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 const uint32_t k_addr = smem_u32(smem + kOffK + st * kTileBytes);
 #pragma unroll
                 for (int ks = 0; ks < kD / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    umma_ss(tmem_base + kColS + sb * 128, smem_desc(q_addr + off, 16, 1024),
-                            smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                    umma_ss(tmem_base + kColS + sb * kTN,
+                            smem_desc(q_addr + (ks >> 2) * kQHalfBytes + (ks & 3) * 32, 16, 1024),
+                            smem_desc(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024), idesc_s, ks > 0);
                 }
                 tc_commit(&s_full[sb]);
                 tc_commit(&k_empty[st]);
@@ -324,26 +370,27 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             ok = __all_sync(kFull, mbar_wait(&s_full[sb], (j >> 1) & 1, p.status));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t s_addr = lane_addr + kColS + sb * 128;
+            const uint32_t s_addr = lane_addr + kColS + sb * kTN;
 
-            // ---- scores of the row for the tile's 128 keys (Eq. 3), their maximum
-            float sc[kTN];
-            float m_tile = -INFINITY;
+            // ---- pass 1: the row's scores for the tile's 128 keys (Eq. 3), only their maximum is kept.  The
+            // loops over the four 32-key chunks are not unrolled: with one warp per scheduler the code has to
+            // stay inside the instruction cache.
             const bool masked = j0 + kTN - 1 > pos;
             const float bias0 = fmaf(slope2, (float)j0, c_row);       // ALiBi term of the tile's first key
-#pragma unroll
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
             for (int c = 0; c < kTN / 32; ++c) {
                 float v[32];
                 tmem_ld32(s_addr + c * 32, v);
+                const float bias_c = fmaf(slope2, (float)(c * 32), bias0);
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    const int jj = j0 + c * 32 + e;
-                    float t = fmaf(v[e], qscale, fmaf(slope2, (float)(c * 32 + e), bias0));
-                    if (masked) t = jj <= pos ? t : -INFINITY;
-                    sc[c * 32 + e] = t;
-                    m_tile = fmaxf(m_tile, t);
+                    float t = fmaf(v[e], qscale, fmaf(slope2, (float)e, bias_c));
+                    if (masked) t = j0 + c * 32 + e <= pos ? t : -INFINITY;
+                    mx[e & 3] = fmaxf(mx[e & 3], t);
                 }
             }
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 
             // ---- running maximum: move it (and rescale l and O) only when it grew by more than the threshold
             // (true for the first tile in which the row sees a key: m_used = -inf until then)
@@ -368,21 +415,33 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             m_used = m_new;
             l *= f;
 
-            // ---- p = 2^(s - m) (Eq. 4), rounded to bf16 pairs over the first 64 columns of S
+            // ---- pass 2: p = 2^(s - m) (Eq. 4) from the scores read again, rounded to bf16 pairs over the first
+            // 64 columns of S: chunk c's 16 columns of P lie below the S columns still to be read
             // (a row that has not seen a key yet has only -inf scores: subtract 0 so that they give p = 0)
             const float m_sub = m_used == -INFINITY ? 0.f : m_used;
-            float sum = 0.f;
+            const float bias_m = bias0 - m_sub;
+            float sm[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+            for (int c = 0; c < kTN / 32; ++c) {
+                float v[32];
+                uint32_t w[16];
+                tmem_ld32(s_addr + c * 32, v);
+                const float bias_c = fmaf(slope2, (float)(c * 32), bias_m);
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t w[32];
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float p0 = ex2(sc[c * 64 + 2 * e] - m_sub), p1 = ex2(sc[c * 64 + 2 * e + 1] - m_sub);
-                    sum += p0 + p1;
+                for (int e = 0; e < 16; ++e) {
+                    float t0 = fmaf(v[2 * e], qscale, fmaf(slope2, (float)(2 * e), bias_c));
+                    float t1 = fmaf(v[2 * e + 1], qscale, fmaf(slope2, (float)(2 * e + 1), bias_c));
+                    if (masked) {
+                        t0 = j0 + c * 32 + 2 * e <= pos ? t0 : -INFINITY;
+                        t1 = j0 + c * 32 + 2 * e + 1 <= pos ? t1 : -INFINITY;
+                    }
+                    const float p0 = ex2(t0), p1 = ex2(t1);
+                    sm[e & 3] += p0 + p1;
                     w[e] = pack2(p0, p1);
                 }
-                tmem_st32(s_addr + c * 32, w);
+                tmem_st16(s_addr + c * 16, w);
             }
+            const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
             l += sum;
 
             if (j0 + kTN > n) {
@@ -391,7 +450,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 const int st = j % kKvStages;
                 ok = __all_sync(kFull, mbar_wait(&v_full[st], (j / kKvStages) & 1, p.status));
                 if (!ok) break;
-                if (j0 + r >= n) {
+                if (r < kTN && j0 + r >= n) {
                     char* vrow = smem + kOffV + st * kTileBytes + r * 128;
 #pragma unroll
                     for (int b = 0; b < 2; ++b)
