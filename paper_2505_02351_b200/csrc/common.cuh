@@ -53,11 +53,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // the timeout and returns false.  The bound is on elapsed time, not on the number of polls: one try_wait may
 // itself block for a while before it reports failure.
 constexpr long long kWaitLimitCycles = 1ll << 28;
+// try_wait that lets the hardware park the warp for up to `ns` nanoseconds while the phase is pending, so that a
+// waiting warp does not take issue slots from the warps it is waiting for.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t ns) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return done != 0;
+}
+
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     do {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_parked(bar, parity, 4000)) return true;
     } while (clock64() - start < kWaitLimitCycles);
     atomicExch(status, OPT_GQA_ERR_TIMEOUT);
     return false;

@@ -203,9 +203,51 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// max of three (one instruction on sm_100)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// Pass 1 over one 32-key chunk of a row's scores: t = s*qscale + slope*(key index) + bias_c, running maxima.
+// kMasked adds the causal select (keys after `pos` count as -inf); tiles left of the diagonal skip it.
+template <bool kMasked>
+__device__ __forceinline__ void chunk_max(const float (&v)[32], float qscale, float slope2, float bias_c, int key0,
+                                          int pos, float (&mx)[4]) {
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        float t0 = fmaf(v[e], qscale, fmaf(slope2, (float)e, bias_c));
+        float t1 = fmaf(v[e + 1], qscale, fmaf(slope2, (float)(e + 1), bias_c));
+        if (kMasked) {
+            t0 = key0 + e <= pos ? t0 : -INFINITY;
+            t1 = key0 + e + 1 <= pos ? t1 : -INFINITY;
+        }
+        mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], t0, t1);
+    }
+}
+
+// Pass 2 over one chunk: p = 2^t (the maximum is folded into bias_c), bf16 pairs for the tensor core, partial sums.
+template <bool kMasked>
+__device__ __forceinline__ void chunk_exp(const float (&v)[32], float qscale, float slope2, float bias_c, int key0,
+                                          int pos, float (&sm)[4], uint32_t (&w)[16]) {
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        float t0 = fmaf(v[2 * e], qscale, fmaf(slope2, (float)(2 * e), bias_c));
+        float t1 = fmaf(v[2 * e + 1], qscale, fmaf(slope2, (float)(2 * e + 1), bias_c));
+        if (kMasked) {
+            t0 = key0 + 2 * e <= pos ? t0 : -INFINITY;
+            t1 = key0 + 2 * e + 1 <= pos ? t1 : -INFINITY;
+        }
+        const float p0 = ex2(t0), p1 = ex2(t1);
+        sm[e & 3] += p0 + p1;
+        w[e] = pack2(p0, p1);
+    }
 }
 
 template <int G>
@@ -375,7 +417,8 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // ---- pass 1: the row's scores for the tile's 128 keys (Eq. 3), only their maximum is kept.  The
             // loops over the four 32-key chunks are not unrolled: with one warp per scheduler the code has to
             // stay inside the instruction cache.
-            const bool masked = j0 + kTN - 1 > pos;
+            // Only tiles on the diagonal need the causal select; the choice is made per warp.
+            const bool masked = __any_sync(kFull, j0 + kTN - 1 > pos);
             const float bias0 = fmaf(slope2, (float)j0, c_row);       // ALiBi term of the tile's first key
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
@@ -383,12 +426,8 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 float v[32];
                 tmem_ld32(s_addr + c * 32, v);
                 const float bias_c = fmaf(slope2, (float)(c * 32), bias0);
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    float t = fmaf(v[e], qscale, fmaf(slope2, (float)e, bias_c));
-                    if (masked) t = j0 + c * 32 + e <= pos ? t : -INFINITY;
-                    mx[e & 3] = fmaxf(mx[e & 3], t);
-                }
+                if (masked) chunk_max<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, mx);
+                else chunk_max<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, mx);
             }
             const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 
@@ -427,18 +466,8 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 uint32_t w[16];
                 tmem_ld32(s_addr + c * 32, v);
                 const float bias_c = fmaf(slope2, (float)(c * 32), bias_m);
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    float t0 = fmaf(v[2 * e], qscale, fmaf(slope2, (float)(2 * e), bias_c));
-                    float t1 = fmaf(v[2 * e + 1], qscale, fmaf(slope2, (float)(2 * e + 1), bias_c));
-                    if (masked) {
-                        t0 = j0 + c * 32 + 2 * e <= pos ? t0 : -INFINITY;
-                        t1 = j0 + c * 32 + 2 * e + 1 <= pos ? t1 : -INFINITY;
-                    }
-                    const float p0 = ex2(t0), p1 = ex2(t1);
-                    sm[e & 3] += p0 + p1;
-                    w[e] = pack2(p0, p1);
-                }
+                if (masked) chunk_exp<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, sm, w);
+                else chunk_exp<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, sm, w);
                 tmem_st16(s_addr + c * 16, w);
             }
             const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
