@@ -162,3 +162,39 @@ def test_empty_batch_and_error_codes_on_device_pointers():
         binding.paged_attention_decode(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
                                        d.alibi_slopes, wl.scale, partition_size=20)
     assert e.value.code == -2
+
+
+def test_decode_step_replayed_from_a_cuda_graph():
+    """One step (append -> balanced decode -> reduce, chained by programmatic dependent launches) captured once
+    and replayed on new inputs written into the same buffers."""
+    wl = W.make_custom("graph", "bf16", 32, 4, 128, 16, [1500, 700, 40], seed=27)
+    d = util.DeviceWorkload(wl)
+    P, maxP = 512, 3
+    ws = torch.empty(binding.workspace_bytes(wl.B, wl.Hq, wl.D, maxP), device="cuda:0", dtype=torch.uint8)
+    k0, v0 = d.k_cache.clone(), d.v_cache.clone()
+
+    def step():
+        binding.decode_step(d.out, d.q, d.k_new, d.v_new, d.slot_mapping, d.k_cache, d.v_cache, d.block_tables,
+                            d.context_lens, d.alibi_slopes, wl.scale, partition_size=P, workspace=ws,
+                            max_partitions=maxP, stream=stream)
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        step()                                   # first call outside capture: one-time per-device set-up
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        step()
+    # new values in the same buffers, then replay
+    wl2 = W.make_custom("graph2", "bf16", 32, 4, 128, 16, [1500, 700, 40], seed=28)
+    for name in ("q", "k_new", "v_new", "k_cache", "v_cache", "block_tables", "slot_mapping"):
+        getattr(d, name).copy_(getattr(wl2, name).cuda())
+    d.out.fill_(float("nan"))
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert binding.device_status() == 0
+    want = util.oracle_attention(wl2)
+    got = d.out.double().cpu().numpy()
+    assert np.max(np.abs(got - want)) <= util.TOL["bf16"]
+    del k0, v0
