@@ -228,6 +228,25 @@ int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t*
                                         int Hq, int Hkv, int D, int bs, int64_t num_blocks, int dtype, void* stream);
 
 /*
+ * The prompt branch with empty caches (Algorithms 1 and 2: "Caches are empty" -> "Adjust Q, K, V
+ * for GQA grouping", "Create ALiBi bias", then Eq. 3-5): every sequence attends causally to its own
+ * new tokens, read from contiguous tensors instead of the paged cache.  Token i of sequence s
+ * (row q_start_loc[s] + i) sees keys 0 .. i of that sequence with bias -slope_h*(i - j); query
+ * head h uses K/V head h / G.  The same tcgen05 kernel as opt_gqa_paged_attention_prefill, with
+ * K/V tiles fetched through 3-D tensor maps over k and v.  (Writing k, v into the cache for later
+ * decode steps is opt_gqa_cache_append, before or after this call.)
+ *
+ *   out, q        [total_q_tokens, Hq, D]   bf16, D = 128
+ *   k, v          [total_q_tokens, Hkv, D]  bf16
+ *   q_start_loc   [B+1] int32               prefix sums of the sequences' lengths, device memory
+ *   total_q_tokens, max_q_len               HOST values, as in opt_gqa_paged_attention_prefill
+ *   alibi_slopes  [Hq] fp32 or NULL (causal mask only)
+ */
+int opt_gqa_prompt_attention(void* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,
+                             int total_q_tokens, int max_q_len, const float* alibi_slopes, float scale, int B, int Hq,
+                             int Hkv, int D, int dtype, void* stream);
+
+/*
  * One decode step of the attention layer, Algorithm 2 from "Store reshaped K, V
  * into C_K, C_V" to "Compute context attention with caches": cache_append of the
  * B new tokens (k_new, v_new [B, Hkv, D], slot_mapping [B]), then decode, then --

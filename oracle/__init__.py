@@ -41,6 +41,7 @@ def lib() -> ctypes.CDLL:
         _lib.oracle_paged_attention.restype = ctypes.c_int
         _lib.oracle_partition_partials.restype = ctypes.c_int
         _lib.oracle_reduce.restype = ctypes.c_int
+        _lib.oracle_prompt_attention.restype = ctypes.c_int
         _lib.oracle_alibi_slopes.restype = None
         _lib.oracle_unpage.restype = None
     return _lib
@@ -151,6 +152,24 @@ def reduce(partial_out, partial_lse, context_lens, P: int) -> np.ndarray:
     )
     if rc != 0:
         raise ValueError("max_partitions too small")
+    return out
+
+
+def prompt_attention(q, k, v, q_start_loc, slopes, scale, dtype: str) -> np.ndarray:
+    """Causal attention of every sequence over its own tokens, contiguous q [T,Hq,D], k, v [T,Hkv,D] (empty caches)."""
+    q, k, v = _check_store(q, dtype), _check_store(k, dtype), _check_store(v, dtype)
+    q_start_loc = np.ascontiguousarray(q_start_loc, dtype=np.int32)
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == v.shape == (T, Hkv, D) and q_start_loc[-1] == T
+    if slopes is not None:
+        slopes = np.ascontiguousarray(slopes, dtype=np.float64)
+    out = np.zeros((T, Hq, D), dtype=np.float64)
+    rc = lib().oracle_prompt_attention(_p(out), _p(q), _p(k), _p(v), _p(q_start_loc), _p(slopes),
+                                       ctypes.c_double(scale), ctypes.c_int(q_start_loc.shape[0] - 1),
+                                       ctypes.c_int(Hq), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(DTYPES[dtype]))
+    if rc != 0:
+        raise ValueError("bad shapes")
     return out
 
 

@@ -239,3 +239,50 @@ void oracle_unpage(double* dst, const void* cache, const int32_t* table, int n, 
         for (int d = 0; d < D; ++d) dst[j * D + d] = load_elem(cache, base + d, dtype);
     }
 }
+
+/*
+ * The prompt branch with empty caches (Algorithm 1: "Caches are empty" -> GQA grouping -> "Create ALiBi
+ * bias" / causal mask -> scores, softmax, weighted sum; Eq. 3-5).  q [T, Hq, D], k, v [T, Hkv, D] are
+ * contiguous; sequence s owns rows q_start_loc[s] .. q_start_loc[s+1]-1 and token i of it sees keys
+ * 0 .. i of the same sequence:
+ *   raw_j = scale * <q_i, k_j> - slope_h * (i - j),  w = softmax_j(raw),  out_i = sum_j w_j v_j.
+ * Query head h uses K/V head h / G.
+ */
+int oracle_prompt_attention(double* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,
+                            const double* slopes, double scale, int B, int Hq, int Hkv, int D, int dtype) {
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    const int G = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int s = 0; s < B; ++s) {
+        for (int h = 0; h < Hq; ++h) {
+            const int64_t t0 = q_start_loc[s], len = q_start_loc[s + 1] - q_start_loc[s];
+            const double slope = slopes ? slopes[h] : 0.0;
+            double* raw = (double*)malloc(sizeof(double) * (size_t)(len > 0 ? len : 1));
+            for (int64_t i = 0; i < len; ++i) {
+                const int64_t qo = ((t0 + i) * Hq + h) * (int64_t)D;
+                double mx = -INFINITY;
+                for (int64_t j = 0; j <= i; ++j) {
+                    const int64_t ko = ((t0 + j) * Hkv + h / G) * (int64_t)D;
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d) dot += load_elem(q, qo + d, dtype) * load_elem(k, ko + d, dtype);
+                    raw[j] = scale * dot - slope * (double)(i - j);
+                    if (raw[j] > mx) mx = raw[j];
+                }
+                double denom = 0.0;
+                for (int64_t j = 0; j <= i; ++j) {
+                    raw[j] = exp(raw[j] - mx);
+                    denom += raw[j];
+                }
+                double* o = out + qo;
+                for (int d = 0; d < D; ++d) o[d] = 0.0;
+                for (int64_t j = 0; j <= i; ++j) {
+                    const int64_t vo = ((t0 + j) * Hkv + h / G) * (int64_t)D;
+                    const double w = raw[j] / denom;
+                    for (int d = 0; d < D; ++d) o[d] += w * load_elem(v, vo + d, dtype);
+                }
+            }
+            free(raw);
+        }
+    }
+    return 0;
+}

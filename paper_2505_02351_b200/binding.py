@@ -39,6 +39,7 @@ SIGNATURES = {
                                              _i, _i64, _i, _vp]),
     "opt_gqa_paged_attention_prefill_mma": (_i, [_vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i,
                                                  _i, _i, _i64, _i, _vp]),
+    "opt_gqa_prompt_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _vp, _f, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_decode_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                  _i, _vp, _i, _i, _vp]),
     "opt_gqa_decode_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _f, _i, _i, _i, _i,
@@ -204,6 +205,17 @@ def paged_attention_prefill_mma(out, q, q_start_loc, max_q_len: int, k_cache, v_
                                 alibi_slopes, scale: float, stream=None) -> None:
     _prefill("opt_gqa_paged_attention_prefill_mma", out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables,
              context_lens, alibi_slopes, scale, stream)
+
+
+def prompt_attention(out, q, k, v, q_start_loc, max_q_len: int, alibi_slopes, scale: float, stream=None) -> None:
+    """Causal GQA-ALiBi attention of each sequence over its own new tokens (contiguous k, v; empty caches)."""
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    B = q_start_loc.shape[0] - 1
+    assert q_start_loc.dtype == torch.int32 and k.shape == v.shape and k.shape[0] == T
+    _check(load().opt_gqa_prompt_attention(
+        _ptr(out), _ptr(q), _ptr(k), _ptr(v), _ptr(q_start_loc), T, max_q_len, _ptr(alibi_slopes), scale, B, Hq, Hkv,
+        D, _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_prompt_attention")
 
 
 def step_staging_bytes(B: int, Hq: int, Hkv: int, D: int, max_blocks_per_seq: int, dtype: torch.dtype) -> int:

@@ -205,6 +205,21 @@ int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t*
                            stream);
 }
 
+int opt_gqa_prompt_attention(void* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,
+                             int total_q_tokens, int max_q_len, const float* alibi_slopes, float scale, int B, int Hq,
+                             int Hkv, int D, int dtype, void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, 16) || D != 128) return OPT_GQA_ERR_SHAPE;
+    if (B == 0 || max_q_len == 0 || total_q_tokens == 0) return OPT_GQA_OK;
+    if (!out || !q || !k || !v || !q_start_loc) return OPT_GQA_ERR_NULL;
+    if (!aligned16(out) || !aligned16(q) || !aligned16(k) || !aligned16(v)) return OPT_GQA_ERR_ALIGN;
+    int* status = device_status_ptr();
+    if (!status) return OPT_GQA_ERR_CUDA;
+    return launch_prompt_umma(out, q, k, v, q_start_loc, total_q_tokens, max_q_len, alibi_slopes, scale, B, Hq, Hkv,
+                              status, static_cast<cudaStream_t>(stream));
+}
+
 int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,
                         const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,
                         int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,

@@ -212,4 +212,9 @@ int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, in
                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
                         int bs, int64_t num_blocks, int* device_status, cudaStream_t stream);
 
+// bf16, D = 128: the prompt branch with empty caches (contiguous k, v of the new tokens), same kernel.
+int launch_prompt_umma(void* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,
+                       int total_q_tokens, int max_q_len, const float* alibi_slopes, float scale, int B, int Hq,
+                       int Hkv, int* device_status, cudaStream_t stream);
+
 }  // namespace optgqa

@@ -250,7 +250,10 @@ __device__ __forceinline__ void chunk_exp(const float (&v)[32], float qscale, fl
     }
 }
 
-template <int G>
+// kPaged: K/V come from the paged cache through block_tables (2-D maps over [rows, D]); otherwise from contiguous
+// k, v [tokens, Hkv, D] holding exactly the new tokens (3-D maps; the prompt branch with empty caches, where a
+// sequence's context is its own new tokens).
+template <int G, bool kPaged>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const UmmaParams p) {
@@ -275,7 +278,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int nblk = (qlen + TQ - 1) / TQ;
     if ((int)blockIdx.x >= nblk) return;
     const int qb = nblk - 1 - (int)blockIdx.x;             // the longest-running blocks start first
-    const int n = p.context_lens[s];
+    const int n = kPaged ? p.context_lens[s] : qlen;
     const int i_last = min(qlen, (qb + 1) * TQ) - 1;        // last valid new token of this block
     const int pos_last = n - qlen + i_last;                 // its position; the block sees keys 0 .. pos_last
     const int ntiles = pos_last / kTN + 1;
@@ -316,11 +319,11 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             tma_load_3d(smem + kOffQ, &map_q, 0, kvh * G, qstart + qb * TQ, q_full);
             tma_load_3d(smem + kOffQ + kQHalfBytes, &map_q, 64, kvh * G, qstart + qb * TQ, q_full);
         }
-        const int32_t* table = p.block_tables + (size_t)s * p.max_blocks;
+        const int32_t* table = kPaged ? p.block_tables + (size_t)s * p.max_blocks : nullptr;
         const int sub = lane & 7;                           // lanes 0-7 fetch one 16-token slice each
         auto page_of = [&](int j) -> int {         // j counts processed tiles; the tile is ntiles - 1 - j
             const int tok = (ntiles - 1 - j) * kTN + sub * kSub;
-            return (lane < 8 && tok < n) ? __ldg(table + tok / p.bs) : -1;
+            return (kPaged && lane < 8 && tok < n) ? __ldg(table + tok / p.bs) : -1;
         };
         int page = page_of(0);
         for (int j = 0; j < ntiles; ++j) {
@@ -337,8 +340,13 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             __syncwarp();
             if (lane < nsub) {
                 char* dst = smem + kOffK + st * kTileBytes + sub * (kSub * 128);
-                tma_load_2d(dst, &map_k, 0, row, &k_full[st]);
-                tma_load_2d(dst + kHalfBytes, &map_k, 64, row, &k_full[st]);
+                if (kPaged) {
+                    tma_load_2d(dst, &map_k, 0, row, &k_full[st]);
+                    tma_load_2d(dst + kHalfBytes, &map_k, 64, row, &k_full[st]);
+                } else {
+                    tma_load_3d(dst, &map_k, 0, kvh, qstart + tok, &k_full[st]);
+                    tma_load_3d(dst + kHalfBytes, &map_k, 64, kvh, qstart + tok, &k_full[st]);
+                }
             }
             if (j >= kKvStages) ok = mbar_wait(&v_empty[st], ((j / kKvStages) - 1) & 1, p.status);
             if (!__all_sync(kFull, ok)) break;
@@ -346,8 +354,13 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             __syncwarp();
             if (lane < nsub) {
                 char* dst = smem + kOffV + st * kTileBytes + sub * (kSub * 128);
-                tma_load_2d(dst, &map_v, 0, row, &v_full[st]);
-                tma_load_2d(dst + kHalfBytes, &map_v, 64, row, &v_full[st]);
+                if (kPaged) {
+                    tma_load_2d(dst, &map_v, 0, row, &v_full[st]);
+                    tma_load_2d(dst + kHalfBytes, &map_v, 64, row, &v_full[st]);
+                } else {
+                    tma_load_3d(dst, &map_v, 0, kvh, qstart + tok, &v_full[st]);
+                    tma_load_3d(dst + kHalfBytes, &map_v, 64, kvh, qstart + tok, &v_full[st]);
+                }
             }
             page = page_next;
         }
@@ -578,21 +591,46 @@ bool make_q_map(CUtensorMap* map, const void* q, int tokens, int Hq, int G) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int G>
+// k or v [tokens, Hkv, 128] as a 3-D tensor; a box is 64 dims x one head x 16 tokens.
+bool make_kv_map(CUtensorMap* map, const void* kv, int tokens, int Hkv) {
+    EncodeFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hkv, (cuuint64_t)tokens};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hkv * kD * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)kSub};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(kv), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int G, bool kPaged>
 int launch_one(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& p, int B,
                int max_q_len, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
     if (dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(prefill_umma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(prefill_umma_kernel<G, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBytes) != cudaSuccess)
             return OPT_GQA_ERR_CUDA;
         configured[dev] = true;
     }
     constexpr int TQ = kRows / G;
     dim3 grid((max_q_len + TQ - 1) / TQ, p.Hkv, B);
-    return launch_dependent(prefill_umma_kernel<G>, grid, dim3(kThreads), kSmemBytes, stream, mq, mk, mv, p);
+    return launch_dependent(prefill_umma_kernel<G, kPaged>, grid, dim3(kThreads), kSmemBytes, stream, mq, mk, mv, p);
+}
+
+template <bool kPaged>
+int launch_g(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& p, int B, int G,
+             int max_q_len, cudaStream_t stream) {
+    switch (G) {
+        case 1: return launch_one<1, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+        case 2: return launch_one<2, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+        case 4: return launch_one<4, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+        case 8: return launch_one<8, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+    }
+    return OPT_GQA_ERR_SHAPE;
 }
 
 }  // namespace
@@ -622,13 +660,32 @@ int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, in
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.bs = bs;
-    switch (G) {
-        case 1: return launch_one<1>(mq, mk, mv, p, B, max_q_len, stream);
-        case 2: return launch_one<2>(mq, mk, mv, p, B, max_q_len, stream);
-        case 4: return launch_one<4>(mq, mk, mv, p, B, max_q_len, stream);
-        case 8: return launch_one<8>(mq, mk, mv, p, B, max_q_len, stream);
-    }
-    return OPT_GQA_ERR_SHAPE;
+    return launch_g<true>(mq, mk, mv, p, B, G, max_q_len, stream);
+}
+
+// The prompt branch with empty caches: q [tokens, Hq, 128], k, v [tokens, Hkv, 128] contiguous, causal + ALiBi.
+int launch_prompt_umma(void* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,
+                       int total_q_tokens, int max_q_len, const float* alibi_slopes, float scale, int B, int Hq,
+                       int Hkv, int* device_status, cudaStream_t stream) {
+    if (total_q_tokens <= 0 || B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
+    const int G = Hq / Hkv;
+    CUtensorMap mq, mk, mv;
+    if (!make_q_map(&mq, q, total_q_tokens, Hq, G) || !make_kv_map(&mk, k, total_q_tokens, Hkv) ||
+        !make_kv_map(&mv, v, total_q_tokens, Hkv))
+        return OPT_GQA_ERR_CUDA;
+    UmmaParams p;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.q_start_loc = q_start_loc;
+    p.block_tables = nullptr;
+    p.context_lens = nullptr;
+    p.slopes = alibi_slopes;
+    p.status = device_status;
+    p.scale = scale;
+    p.max_blocks = 0;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.bs = 16;
+    return launch_g<false>(mq, mk, mv, p, B, G, max_q_len, stream);
 }
 
 }  // namespace optgqa

@@ -89,3 +89,48 @@ def test_config5_full_size_sampled_rows():
     assert err <= TOL, err
     # property that holds at any size: every output lies in the convex hull of V's value range
     assert np.abs(got).max() <= float(wl.v_cache.float().abs().max().item()) + float(wl.v_new.float().abs().max().item())
+
+
+# ------------------------------------------------------------------ the prompt branch with empty caches (contiguous k, v)
+def _prompt(wl, slopes=True):
+    import oracle
+    dev = "cuda:0"
+    q, k, v, qsl = wl.q.to(dev), wl.k_new.to(dev), wl.v_new.to(dev), wl.q_start_loc.to(dev)
+    sl = wl.alibi_slopes.to(dev) if slopes else None
+    out = torch.full_like(q, float("nan"))
+    lens = wl.q_start_loc.numpy()[1:] - wl.q_start_loc.numpy()[:-1]
+    binding.prompt_attention(out, q, k, v, qsl, int(lens.max()), sl, wl.scale)
+    torch.cuda.synchronize()
+    assert binding.device_status() == 0
+    want = oracle.prompt_attention(W.storage_numpy(wl.q), W.storage_numpy(wl.k_new), W.storage_numpy(wl.v_new),
+                                   wl.q_start_loc.numpy(), wl.alibi_slopes.numpy().astype(np.float64) if slopes else None,
+                                   wl.scale, "bf16")
+    got = out.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.max(np.abs(got - want)) <= TOL, wl.name
+    return got
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (4, 2), (8, 2), (8, 1), (32, 8)])
+def test_prompt_attention_contiguous(Hq, Hkv):
+    lens = [200, 77, 1, 129, 64, 300, 128]
+    wl = W.make_custom("prompt", "bf16", Hq, Hkv, 128, 16, lens, q_lens=lens, seed=70 + Hq)
+    _prompt(wl)
+    _prompt(wl, slopes=False)
+
+
+def test_prompt_attention_equals_prefill_over_the_appended_cache():
+    lens = [513, 40, 1000]
+    wl = W.make_custom("prompt2", "bf16", 8, 2, 128, 16, lens, q_lens=lens, seed=75)
+    got = _prompt(wl)
+    paged, _ = util.gpu_prefill(wl)           # append the same tokens into pages, then prefill over the pages
+    assert np.array_equal(got, paged)         # same kernel, same tiles, same order: bitwise equal
+
+
+def test_prompt_attention_rejects_what_it_does_not_support():
+    wl = W.make_custom("prompt3", "bf16", 4, 2, 64, 16, [10], q_lens=[10], seed=76)
+    q = wl.q.cuda()
+    with pytest.raises(binding.OptGqaError) as e:
+        binding.prompt_attention(torch.empty_like(q), q, wl.k_new.cuda(), wl.v_new.cuda(), wl.q_start_loc.cuda(), 10,
+                                 None, wl.scale)
+    assert e.value.code == -2                 # head_dim 64 is not built for this entry point

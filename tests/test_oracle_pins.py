@@ -364,3 +364,42 @@ def test_bf16_widening_is_exact():
     cache = W.storage_numpy(x).reshape(1, 1, 5, 1)
     seq = oracle.unpage(cache, np.array([0], np.int32), 5, 0, "bf16")
     assert np.array_equal(seq[:, 0], x.double().numpy())
+
+
+# ------------------------------------------------------------------ the prompt branch with empty caches
+def _prompt_inputs(Hq, Hkv, D, lens, dtype, seed):
+    wl = W.make_custom("prompt", dtype, Hq, Hkv, D, 16, lens, q_lens=lens, seed=seed)
+    return wl, W.storage_numpy(wl.q), W.storage_numpy(wl.k_new), W.storage_numpy(wl.v_new), wl.q_start_loc.numpy()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_prompt_attention_matches_dense_numpy(dtype):
+    """Written out with matrices in numpy, sequence by sequence: softmax(scale QK^T - slope*(i-j), j <= i) V."""
+    wl, q, k, v, qsl = _prompt_inputs(4, 2, 64, [5, 33, 1, 18], dtype, 61)
+    slopes = wl.alibi_slopes.numpy().astype(np.float64)
+    got = oracle.prompt_attention(q, k, v, qsl, slopes, wl.scale, dtype)
+    qd, kd, vd = brute.widen(q), brute.widen(k), brute.widen(v)
+    for s in range(4):
+        a, b = qsl[s], qsl[s + 1]
+        i = np.arange(b - a)
+        rel = i[:, None] - i[None, :]
+        for h in range(4):
+            S = wl.scale * qd[a:b, h] @ kd[a:b, h // 2].T - slopes[h] * rel
+            S = np.where(rel < 0, -np.inf, S)
+            Wt = np.exp(S - S.max(axis=1, keepdims=True))
+            Wt /= Wt.sum(axis=1, keepdims=True)
+            assert np.max(np.abs(got[a:b, h] - Wt @ vd[a:b, h // 2])) < 1e-12
+
+
+def test_prompt_attention_is_prefill_over_a_cache_holding_only_the_new_tokens():
+    wl, q, k, v, qsl = _prompt_inputs(8, 2, 64, [40, 7, 65], "bf16", 62)
+    slopes = wl.alibi_slopes.numpy().astype(np.float64)
+    kc, vc = W.storage_numpy(wl.k_cache), W.storage_numpy(wl.v_cache)
+    oracle.cache_append(k, v, kc, vc, wl.slot_mapping.numpy(), "bf16")
+    paged = oracle.paged_attention(q, kc, vc, wl.block_tables.numpy(), wl.context_lens.numpy(), slopes, wl.scale,
+                                   "bf16", q_start_loc=qsl)
+    got = oracle.prompt_attention(q, k, v, qsl, slopes, wl.scale, "bf16")
+    assert np.max(np.abs(got - paged)) < 1e-12
+    # the first token of every sequence sees only itself
+    for s in range(3):
+        assert np.allclose(got[qsl[s]], brute.widen(v)[qsl[s]].repeat(4, axis=0), atol=1e-15)
