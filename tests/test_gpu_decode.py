@@ -198,3 +198,29 @@ def test_decode_step_replayed_from_a_cuda_graph():
     got = d.out.double().cpu().numpy()
     assert np.max(np.abs(got - want)) <= util.TOL["bf16"]
     del k0, v0
+
+
+def test_one_very_long_sequence():
+    """200k tokens in one sequence (12.5k pages): the stream is cut across all workers, partitions of 512 and 4096."""
+    wl = W.make_custom("long", "bf16", 8, 1, 128, 16, [200_003], seed=29)
+    _check(wl, partition_size=512, balanced=True)
+    _check(wl, partition_size=4096)
+    _check(wl, partition_size=4096, balanced=True)
+
+
+def test_many_short_sequences():
+    """2048 sequences of 0..64 tokens: more sequences than one 32-lane scan step, single-tile pieces, empty rows."""
+    rng = np.random.default_rng(30)
+    lens = rng.integers(0, 65, size=2048)
+    wl = W.make_custom("short", "bf16", 8, 1, 128, 16, lens, seed=30, poison=True)
+    _check(wl, partition_size=512, balanced=True)
+    _check(wl, partition_size=16)
+    _check(wl)
+
+
+def test_largest_group_and_smallest_head_dim():
+    wl = W.make_custom("g8d64", "bf16", 64, 8, 64, 32, [3000, 17, 4100], seed=31, poison=True)
+    _check(wl, partition_size=512, balanced=True)
+    _check(wl, partition_size=256)
+    wl32 = W.make_custom("g8d64f", "fp32", 16, 2, 64, 32, [700, 17], seed=32, poison=True)
+    _check(wl32, partition_size=128)
