@@ -272,8 +272,10 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
  * runs there, and out is copied back to out_host; the call returns once everything
  * is enqueued, so synchronise `stream` before reading out_host or reusing the host
  * buffers.  The cache, alibi_slopes and workspace stay DEVICE pointers: the cache
- * is state that persists between steps.  (Convenience wrapper around the step; the
- * transfers are the "Reshape Q, K, V" hand-over of Algorithm 2's inputs.)
+ * is state that persists between steps.  Page-locked (pinned, mapped) host buffers are
+ * read by one gather kernel and out is stored into out_host by the step's last kernel;
+ * pageable buffers are moved with cudaMemcpyAsync instead.  (Convenience wrapper around the
+ * step; the transfers are the "Reshape Q, K, V" hand-over of Algorithm 2's inputs.)
  */
 int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_new_host, const void* v_new_host,
                              const int64_t* slot_mapping_host, const int32_t* block_tables_host,

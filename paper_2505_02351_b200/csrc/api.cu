@@ -251,6 +251,32 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
 }
 
 namespace {
+// Six host arrays copied to device staging by ONE kernel that reads pinned host memory directly (32-bit words).
+struct HostGather {
+    const uint32_t* src[6];
+    uint32_t* dst[6];
+    unsigned words[6];
+};
+
+__global__ void __launch_bounds__(256) gather_host_kernel(const HostGather g) {
+    const unsigned tid = blockIdx.x * blockDim.x + threadIdx.x, nthreads = gridDim.x * blockDim.x;
+#pragma unroll
+    for (int a = 0; a < 6; ++a)
+        for (unsigned i = tid; i < g.words[a]; i += nthreads) g.dst[a][i] = g.src[a][i];
+}
+
+// The device-side address of pinned (page-locked, mapped) host memory, or nullptr for pageable memory.
+const void* device_view(const void* host) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    if (attr.type != cudaMemoryTypeHost || !attr.devicePointer) return nullptr;
+    if (reinterpret_cast<uintptr_t>(attr.devicePointer) & 3u) return nullptr;
+    return attr.devicePointer;
+}
+
 struct StagingLayout {
     size_t q, k_new, v_new, out, slots, tables, lens, total;
 };
@@ -295,22 +321,40 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
     char* st = static_cast<char*>(staging);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const size_t qb = (size_t)B * Hq * D * es, kb = (size_t)B * Hkv * D * es;
-    bool ok = true;
-    ok &= cudaMemcpyAsync(st + L.q, q_host, qb, cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    ok &= cudaMemcpyAsync(st + L.k_new, k_new_host, kb, cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    ok &= cudaMemcpyAsync(st + L.v_new, v_new_host, kb, cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    ok &= cudaMemcpyAsync(st + L.slots, slot_mapping_host, (size_t)B * 8, cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    ok &= cudaMemcpyAsync(st + L.tables, block_tables_host, (size_t)B * max_blocks_per_seq * 4,
-                          cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    ok &= cudaMemcpyAsync(st + L.lens, context_lens_host, (size_t)B * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
-    if (!ok) return OPT_GQA_ERR_CUDA;
-    int rc = opt_gqa_decode_step(st + L.out, st + L.q, st + L.k_new, st + L.v_new,
+    // Pinned host buffers are read and written by the kernels themselves: one gather kernel instead of six copies,
+    // and the last kernel of the step stores out straight into out_host.  Pageable buffers go through
+    // cudaMemcpyAsync.
+    const void* src[6] = {q_host, k_new_host, v_new_host, slot_mapping_host, block_tables_host, context_lens_host};
+    const size_t off[6] = {L.q, L.k_new, L.v_new, L.slots, L.tables, L.lens};
+    const size_t bytes[6] = {qb, kb, kb, (size_t)B * 8, (size_t)B * max_blocks_per_seq * 4, (size_t)B * 4};
+    HostGather g;
+    bool pinned = true;
+    for (int a = 0; a < 6; ++a) {
+        const void* dv = device_view(src[a]);
+        pinned &= dv != nullptr && bytes[a] % 4 == 0 && bytes[a] / 4 <= 0xffffffffull;
+        g.src[a] = static_cast<const uint32_t*>(dv);
+        g.dst[a] = reinterpret_cast<uint32_t*>(st + off[a]);
+        g.words[a] = (unsigned)(bytes[a] / 4);
+    }
+    void* out_dev = pinned ? const_cast<void*>(device_view(out_host)) : nullptr;
+    pinned &= out_dev != nullptr && (reinterpret_cast<uintptr_t>(out_dev) & 15u) == 0;
+    if (pinned) {
+        gather_host_kernel<<<32, 256, 0, cs>>>(g);
+        if (cudaGetLastError() != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    } else {
+        bool ok = true;
+        for (int a = 0; a < 6; ++a)
+            ok &= cudaMemcpyAsync(st + off[a], src[a], bytes[a], cudaMemcpyHostToDevice, cs) == cudaSuccess;
+        if (!ok) return OPT_GQA_ERR_CUDA;
+    }
+    int rc = opt_gqa_decode_step(pinned ? out_dev : st + L.out, st + L.q, st + L.k_new, st + L.v_new,
                                  reinterpret_cast<const int64_t*>(st + L.slots), k_cache, v_cache,
                                  reinterpret_cast<const int32_t*>(st + L.tables), max_blocks_per_seq,
                                  reinterpret_cast<const int32_t*>(st + L.lens), alibi_slopes, scale, B, Hq, Hkv, D,
                                  bs, num_blocks, partition_size, workspace, max_partitions, dtype, stream);
     if (rc != OPT_GQA_OK) return rc;
-    if (cudaMemcpyAsync(out_host, st + L.out, qb, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return OPT_GQA_ERR_CUDA;
+    if (!pinned && cudaMemcpyAsync(out_host, st + L.out, qb, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+        return OPT_GQA_ERR_CUDA;
     return OPT_GQA_OK;
 }
 

@@ -224,3 +224,25 @@ def test_largest_group_and_smallest_head_dim():
     _check(wl, partition_size=256)
     wl32 = W.make_custom("g8d64f", "fp32", 16, 2, 64, 32, [700, 17], seed=32, poison=True)
     _check(wl32, partition_size=128)
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_from_host_buffers(pinned):
+    """opt_gqa_decode_step_host: pinned buffers are read and written by the kernels directly, pageable ones are copied."""
+    for wl, P in ((W.make_config(3, shrink=8), 512), (W.make_config(1), 0)):
+        d = util.DeviceWorkload(wl)
+        pin = (lambda t: t.contiguous().pin_memory()) if pinned else (lambda t: t.contiguous().clone())
+        hq, hk, hv = pin(wl.q), pin(wl.k_new), pin(wl.v_new)
+        hs, ht, hl = pin(wl.slot_mapping), pin(wl.block_tables), pin(wl.context_lens)
+        hout = pin(torch.full_like(wl.q, float("nan")))
+        tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+        maxP = max(1, (int(wl.context_lens.max()) + P - 1) // P) if P else 1
+        staging = torch.empty(binding.step_staging_bytes(wl.B, wl.Hq, wl.Hkv, wl.D, wl.max_blocks, tdt), dtype=torch.uint8,
+                              device="cuda:0")
+        ws = torch.empty(max(16, binding.workspace_bytes(wl.B, wl.Hq, wl.D, maxP)), dtype=torch.uint8, device="cuda:0")
+        binding.decode_step_host(hout, hq, hk, hv, hs, ht, hl, staging, d.k_cache, d.v_cache, d.alibi_slopes, wl.scale,
+                                 partition_size=P, workspace=ws if P else None, max_partitions=maxP)
+        torch.cuda.synchronize()
+        assert binding.device_status() == 0
+        want = util.oracle_attention(wl)
+        assert np.max(np.abs(hout.double().numpy() - want)) <= util.TOL[wl.dtype], (wl.name, pinned)
