@@ -22,9 +22,7 @@
 //   O^T += V^T p^T           one m16n8k16 per 16 output dims            (Eq. 5)
 // p^T reaches its operand layout through movmatrix; the denominator sums the same
 // rounded p that the tensor core multiplies; accumulation is fp32.
-#include <cuda.h>
-
-#include "common.cuh"
+#include "tma_mma.cuh"
 
 namespace optgqa {
 
@@ -77,39 +75,11 @@ struct StreamCfg {
     static constexpr int SMEM = OFF_BAR + kWarps * kStages * 8 + 1024;   // + slack to align the ring to 1 KB
 };
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-            smem_u32(dst)),
-        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
-        : "memory");
-}
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-
 // Transposes an 8x8 matrix of 16-bit elements held one row pair per thread (the ldmatrix layout).
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     uint32_t d;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
-}
-
-// d += a * b, m16n8k16, bf16 operands, fp32 accumulate.
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 // Byte offset of 16-byte chunk `chunk` (0 .. D/8-1) of token row `row` inside a tile stored as
@@ -509,36 +479,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     }
 }
 
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn() {
-    static EncodeFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeFn>(p);
-    }
-    return fn;
-}
-
-// The cache seen as a 2-D bf16 tensor [num_blocks*Hkv*bs rows, D]; a box is 16 token rows x 64 dims (128 B).
-bool make_map(CUtensorMap* map, const void* cache, uint64_t rows, int D) {
-    EncodeFn enc = encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kTileTok};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 int sm_count() {
     static int counts[64] = {};
     int dev = 0;
@@ -593,7 +533,8 @@ int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
     CUtensorMap mk, mv;
-    if (!make_map(&mk, k_cache, rows, D) || !make_map(&mv, v_cache, rows, D)) return OPT_GQA_ERR_CUDA;
+    if (!make_cache_map(&mk, k_cache, rows, D, kTileTok) || !make_cache_map(&mv, v_cache, rows, D, kTileTok))
+        return OPT_GQA_ERR_CUDA;
     StreamParams p;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.block_tables = block_tables;

@@ -15,9 +15,7 @@
 // (B operand of p V) bank-conflict free.  Scores stay in fp32 registers; p is
 // rounded to bf16 only as the tensor-core operand and the denominator sums the same
 // rounded values; accumulation is fp32.
-#include <cuda.h>
-
-#include "common.cuh"
+#include "tma_mma.cuh"
 
 namespace optgqa {
 
@@ -69,28 +67,8 @@ struct TcCfg {
     static_assert(G * D * 4 <= WARP_RING, "merge buffer must fit in the warp's ring");
 };
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-            smem_u32(dst)),
-        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
-        : "memory");
-}
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-
 // d += a * b, m16n8k16, bf16 operands, fp32 accumulate.  Rows 8..15 of a are zero here (a1 = a3 = 0).
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_bf16_rows8(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
@@ -231,8 +209,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             for (int ks = 0; ks < KS; ++ks) {
                 uint32_t b[4];
                 ldmatrix_x4(b, kbase + swz(krow, 2 * ks + (lmat & 1)));
-                mma_bf16(sa, qa[ks][0], qa[ks][1], b[0], b[1]);
-                mma_bf16(sb, qa[ks][0], qa[ks][1], b[2], b[3]);
+                mma_bf16_rows8(sa, qa[ks][0], qa[ks][1], b[0], b[1]);
+                mma_bf16_rows8(sb, qa[ks][0], qa[ks][1], b[2], b[3]);
             }
         }
         // thread holds head g, tokens j0 + {2t, 2t+1} (sa[0], sa[1]) and j0 + 8 + {2t, 2t+1} (sb[0], sb[1])
@@ -279,8 +257,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             for (int jj = 0; jj < NT / 2; ++jj) {
                 uint32_t b[4];
                 ldmatrix_x4_trans(b, vbase + swz(vrow, 2 * jj + (lmat >> 1)));
-                mma_bf16(o[2 * jj], pa0, pa2, b[0], b[1]);
-                mma_bf16(o[2 * jj + 1], pa0, pa2, b[2], b[3]);
+                mma_bf16_rows8(o[2 * jj], pa0, pa2, b[0], b[1]);
+                mma_bf16_rows8(o[2 * jj + 1], pa0, pa2, b[2], b[3]);
             }
         }
 
@@ -331,36 +309,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     }
 }
 
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn() {
-    static EncodeFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeFn>(p);
-    }
-    return fn;
-}
-
-// The cache seen as a 2-D bf16 tensor [num_blocks*Hkv*bs rows, D]; a box is 16 token rows x 64 dims (128 B).
-bool make_map(CUtensorMap* map, const void* cache, uint64_t rows, int D) {
-    EncodeFn enc = encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kTileTok};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int D, int G>
 int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, int B, cudaStream_t stream) {
     using C = TcCfg<D, G>;
@@ -397,7 +345,8 @@ int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* 
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
     CUtensorMap mk, mv;
-    if (!make_map(&mk, k_cache, rows, D) || !make_map(&mv, v_cache, rows, D)) return OPT_GQA_ERR_CUDA;
+    if (!make_cache_map(&mk, k_cache, rows, D, kTileTok) || !make_cache_map(&mv, v_cache, rows, D, kTileTok))
+        return OPT_GQA_ERR_CUDA;
     TcParams p;
     p.out = out;
     p.q = static_cast<const __nv_bfloat16*>(q);

@@ -23,9 +23,7 @@
 // default shape is 64-key tiles in a two-stage ring: two CTAs fit on an SM (96 KiB of shared memory
 // and 256 tensor-memory columns each) and one CTA's exp2 phase overlaps the other's maximum phase.
 // Every wait is a bounded mbarrier wait.
-#include <cuda.h>
-
-#include "common.cuh"
+#include "tma_mma.cuh"
 
 namespace optgqa {
 
@@ -83,26 +81,6 @@ struct UmmaParams {
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-            smem_u32(dst)),
-        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
-        : "memory");
-}
-
-__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
-            smem_u32(dst)),
-        "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
-        : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -547,61 +525,21 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
 }
 
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn() {
-    static EncodeFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeFn>(p);
-    }
-    return fn;
-}
-
-// The cache seen as a 2-D bf16 tensor [num_blocks*Hkv*bs rows, 128]; a box is 16 token rows x 64 dims (128 B).
-bool make_cache_map(CUtensorMap* map, const void* cache, uint64_t rows) {
-    EncodeFn enc = encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kSub};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // q [tokens, Hq, 128] as a 3-D tensor; a box is 64 dims x the G heads of a group x 128 / G tokens, i.e. one
 // 64-dim half of the CTA's 128 rows, head-fastest.  Tokens past the end of q read as zeros.
 bool make_q_map(CUtensorMap* map, const void* q, int tokens, int Hq, int G) {
-    EncodeFn enc = encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hq, (cuuint64_t)tokens};
-    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hq * kD * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(kRows / G)};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hq, (cuuint64_t)tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hq * kD * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(kRows / G)};
+    return make_bf16_map(map, q, 3, dims, strides, box);
 }
 
 // k or v [tokens, Hkv, 128] as a 3-D tensor; a box is 64 dims x one head x 16 tokens.
 bool make_kv_map(CUtensorMap* map, const void* kv, int tokens, int Hkv) {
-    EncodeFn enc = encode_fn();
-    if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hkv, (cuuint64_t)tokens};
-    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hkv * kD * 2};
-    cuuint32_t box[3] = {64, 1, (cuuint32_t)kSub};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(kv), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hkv, (cuuint64_t)tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hkv * kD * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kSub};
+    return make_bf16_map(map, kv, 3, dims, strides, box);
 }
 
 template <int G, bool kPaged>
@@ -645,8 +583,8 @@ int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, in
     if (B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
     const int G = Hq / Hkv;
     CUtensorMap mq, mk, mv;
-    if (!make_q_map(&mq, q, total_q_tokens, Hq, G) || !make_cache_map(&mk, k_cache, rows) ||
-        !make_cache_map(&mv, v_cache, rows))
+    if (!make_q_map(&mq, q, total_q_tokens, Hq, G) || !make_cache_map(&mk, k_cache, rows, kD, kSub) ||
+        !make_cache_map(&mv, v_cache, rows, kD, kSub))
         return OPT_GQA_ERR_CUDA;
     UmmaParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
