@@ -228,6 +228,32 @@ int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t*
                                         int Hq, int Hkv, int D, int bs, int64_t num_blocks, int dtype, void* stream);
 
 /*
+ * Decode and chunked prefill with a local (sliding-window) mask: Algorithm 1, "Create causal and
+ * local attention masks" -- the branch taken when no ALiBi slopes are given, although slopes are
+ * accepted here as well.  The token at position pos attends to keys pos - window < j <= pos only;
+ * everything else is as in Eq. 3-5.  Neither mask exists in memory: the window moves the first tile
+ * a sequence's stream (or a query block's key range) starts at, and the edge tile is masked from the
+ * indices.
+ *
+ * opt_gqa_paged_attention_decode_local: the balanced split and its merge in one call (arguments as
+ * opt_gqa_paged_attention_decode_balanced followed by opt_gqa_paged_attention_reduce_balanced; out
+ * [B, Hq, D] is written; bf16 caches, partition_size > 0).  opt_gqa_paged_attention_prefill_local:
+ * arguments as opt_gqa_paged_attention_prefill (bf16, D = 128).  window > 0 is required.
+ */
+int opt_gqa_paged_attention_decode_local(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                         const int32_t* block_tables, int max_blocks_per_seq,
+                                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                         int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                                         void* workspace, int max_partitions, int window, int dtype, void* stream);
+
+int opt_gqa_paged_attention_prefill_local(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+                                          int max_q_len, const void* k_cache, const void* v_cache,
+                                          const int32_t* block_tables, int max_blocks_per_seq,
+                                          const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                          int Hq, int Hkv, int D, int bs, int64_t num_blocks, int window, int dtype,
+                                          void* stream);
+
+/*
  * The prompt branch with empty caches (Algorithms 1 and 2: "Caches are empty" -> "Adjust Q, K, V
  * for GQA grouping", "Create ALiBi bias", then Eq. 3-5): every sequence attends causally to its own
  * new tokens, read from contiguous tensors instead of the paged cache.  Token i of sequence s

@@ -39,6 +39,10 @@ SIGNATURES = {
                                              _i, _i64, _i, _vp]),
     "opt_gqa_paged_attention_prefill_mma": (_i, [_vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i,
                                                  _i, _i, _i64, _i, _vp]),
+    "opt_gqa_paged_attention_decode_local": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
+                                                  _i, _vp, _i, _i, _i, _vp]),
+    "opt_gqa_paged_attention_prefill_local": (_i, [_vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i,
+                                                   _i, _i, _i64, _i, _i, _vp]),
     "opt_gqa_prompt_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _vp, _f, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_decode_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                  _i, _vp, _i, _i, _vp]),
@@ -205,6 +209,29 @@ def paged_attention_prefill_mma(out, q, q_start_loc, max_q_len: int, k_cache, v_
                                 alibi_slopes, scale: float, stream=None) -> None:
     _prefill("opt_gqa_paged_attention_prefill_mma", out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables,
              context_lens, alibi_slopes, scale, stream)
+
+
+def paged_attention_decode_local(out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
+                                 partition_size: int, workspace, max_partitions: int, window: int, stream=None) -> None:
+    """Balanced decode + merge where every query sees only the last `window` keys of its sequence."""
+    B, Hq, D = q.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    _check(load().opt_gqa_paged_attention_decode_local(
+        _ptr(out), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables), block_tables.shape[1],
+        _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, _ptr(workspace),
+        max_partitions, window, _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_decode_local")
+
+
+def paged_attention_prefill_local(out, q, q_start_loc, max_q_len: int, k_cache, v_cache, block_tables, context_lens,
+                                  alibi_slopes, scale: float, window: int, stream=None) -> None:
+    """Chunked prefill where the token at pos sees keys pos - window < j <= pos."""
+    T, Hq, D = q.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    B = context_lens.shape[0]
+    _check(load().opt_gqa_paged_attention_prefill_local(
+        _ptr(out), _ptr(q), _ptr(q_start_loc), T, max_q_len, _ptr(k_cache), _ptr(v_cache), _ptr(block_tables),
+        block_tables.shape[1], _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, window,
+        _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_prefill_local")
 
 
 def prompt_attention(out, q, k, v, q_start_loc, max_q_len: int, alibi_slopes, scale: float, stream=None) -> None:

@@ -77,7 +77,7 @@ static int decode_checked(bool allow_tensor_cores, void* out, const void* q, con
     if (allow_tensor_cores && dtype == OPT_GQA_BF16 && partition_size > 0)
         return launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
                                     scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out, partial_lse,
-                                    nullptr, max_partitions, status, cs);
+                                    nullptr, max_partitions, 0, status, cs);
     if (allow_tensor_cores && dtype == OPT_GQA_BF16)
         return launch_decode_tc(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                                 alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
@@ -123,16 +123,15 @@ int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const fl
                          dtype, static_cast<cudaStream_t>(stream));
 }
 
-int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, const void* v_cache,
-                                            const int32_t* block_tables, int max_blocks_per_seq,
-                                            const int32_t* context_lens, const float* alibi_slopes, float scale,
-                                            int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
-                                            int partition_size, void* workspace, int max_partitions, int dtype,
-                                            void* stream) {
+static int decode_balanced_checked(const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
+                                   const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
+                                   int64_t num_blocks, int partition_size, void* workspace, int max_partitions,
+                                   int window, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0 || partition_size <= 0 ||
-        partition_size % 16 != 0 || max_partitions <= 0)
+        partition_size % 16 != 0 || max_partitions <= 0 || window < 0)
         return OPT_GQA_ERR_SHAPE;
     if (B > 65535 || Hkv > 65535 || max_partitions > 65535) return OPT_GQA_ERR_SHAPE;
     if (B == 0) return OPT_GQA_OK;
@@ -143,24 +142,57 @@ int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, 
     if (!status) return OPT_GQA_ERR_CUDA;
     return launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
                                 scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, nullptr, nullptr, workspace,
-                                max_partitions, status, static_cast<cudaStream_t>(stream));
+                                max_partitions, window, status, static_cast<cudaStream_t>(stream));
+}
+
+int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, const void* v_cache,
+                                            const int32_t* block_tables, int max_blocks_per_seq,
+                                            const int32_t* context_lens, const float* alibi_slopes, float scale,
+                                            int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
+                                            int partition_size, void* workspace, int max_partitions, int dtype,
+                                            void* stream) {
+    return decode_balanced_checked(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
+                                   scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, max_partitions, 0,
+                                   dtype, stream);
+}
+
+static int reduce_balanced_checked(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq,
+                                   int Hkv, int D, int partition_size, int max_partitions, int window, int dtype,
+                                   void* stream) {
+    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128) || partition_size <= 0 ||
+        partition_size % 16 != 0 || max_partitions <= 0 || window < 0)
+        return OPT_GQA_ERR_SHAPE;
+    if (B == 0) return OPT_GQA_OK;
+    if (!out || !workspace || !context_lens) return OPT_GQA_ERR_NULL;
+    if (!aligned16(out) || !aligned16(workspace)) return OPT_GQA_ERR_ALIGN;
+    return launch_reduce_balanced(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, window,
+                                  dtype, static_cast<cudaStream_t>(stream));
 }
 
 int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B,
                                             int Hq, int Hkv, int D, int partition_size, int max_partitions,
                                             int dtype, void* stream) {
-    if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
-    if (B < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128) || partition_size <= 0 ||
-        partition_size % 16 != 0 || max_partitions <= 0)
-        return OPT_GQA_ERR_SHAPE;
-    if (B == 0) return OPT_GQA_OK;
-    if (!out || !workspace || !context_lens) return OPT_GQA_ERR_NULL;
-    if (!aligned16(out) || !aligned16(workspace)) return OPT_GQA_ERR_ALIGN;
-    return launch_reduce_balanced(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, dtype,
-                                  static_cast<cudaStream_t>(stream));
+    return reduce_balanced_checked(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, 0, dtype,
+                                   stream);
 }
 
-static int prefill_checked(bool allow_umma, void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+int opt_gqa_paged_attention_decode_local(void* out, const void* q, const void* k_cache, const void* v_cache,
+                                         const int32_t* block_tables, int max_blocks_per_seq,
+                                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                         int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                                         void* workspace, int max_partitions, int window, int dtype, void* stream) {
+    if (window <= 0) return OPT_GQA_ERR_SHAPE;
+    if (B > 0 && !out) return OPT_GQA_ERR_NULL;
+    int rc = decode_balanced_checked(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
+                                     scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, max_partitions,
+                                     window, dtype, stream);
+    if (rc != OPT_GQA_OK || B == 0) return rc;
+    return reduce_balanced_checked(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, window,
+                                   dtype, stream);
+}
+
+static int prefill_checked(bool allow_umma, int window, void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
                            int max_q_len, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                            int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,
                            float scale, int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int dtype,
@@ -168,7 +200,7 @@ static int prefill_checked(bool allow_umma, void* out, const void* q, const int3
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 ||
-        num_blocks < 0)
+        num_blocks < 0 || window < 0 || (window > 0 && !(allow_umma && D == 128)))
         return OPT_GQA_ERR_SHAPE;
     if (B == 0 || max_q_len == 0 || total_q_tokens == 0) return OPT_GQA_OK;
     if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
@@ -179,7 +211,7 @@ static int prefill_checked(bool allow_umma, void* out, const void* q, const int3
     if (allow_umma && D == 128)
         return launch_prefill_umma(out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
                                    max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, bs, num_blocks,
-                                   status, static_cast<cudaStream_t>(stream));
+                                   window, status, static_cast<cudaStream_t>(stream));
     return launch_prefill(out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables, max_blocks_per_seq,
                           context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, status,
                           static_cast<cudaStream_t>(stream));
@@ -190,7 +222,7 @@ int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_s
                                     const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
                                     const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
                                     int64_t num_blocks, int dtype, void* stream) {
-    return prefill_checked(true, out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
+    return prefill_checked(true, 0, out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
                            max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, dtype,
                            stream);
 }
@@ -200,7 +232,19 @@ int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t*
                                         const int32_t* block_tables, int max_blocks_per_seq,
                                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
                                         int Hq, int Hkv, int D, int bs, int64_t num_blocks, int dtype, void* stream) {
-    return prefill_checked(false, out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
+    return prefill_checked(false, 0, out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
+                           max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, dtype,
+                           stream);
+}
+
+int opt_gqa_paged_attention_prefill_local(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
+                                          int max_q_len, const void* k_cache, const void* v_cache,
+                                          const int32_t* block_tables, int max_blocks_per_seq,
+                                          const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
+                                          int Hq, int Hkv, int D, int bs, int64_t num_blocks, int window, int dtype,
+                                          void* stream) {
+    if (window <= 0) return OPT_GQA_ERR_SHAPE;
+    return prefill_checked(true, window, out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
                            max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, dtype,
                            stream);
 }

@@ -191,12 +191,12 @@ inline BalancedLayout balanced_layout(int B, int Hq, int Hkv, int D, int max_par
 int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                          int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                         float* partial_out, float* partial_lse, void* workspace, int max_partitions,
+                         float* partial_out, float* partial_lse, void* workspace, int max_partitions, int window,
                          int* device_status, cudaStream_t stream);
 
 // Merge of the balanced split's pieces (reduce.cu).
 int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
-                           int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream);
+                           int D, int partition_size, int max_partitions, int window, int dtype, cudaStream_t stream);
 
 int launch_reduce(void* out, const float* partial_out, const float* partial_lse, const int32_t* context_lens,
                   int B, int Hq, int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream);
@@ -210,7 +210,7 @@ int launch_prefill(void* out, const void* q, const int32_t* q_start_loc, int max
 int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens, int max_q_len,
                         const void* k_cache, const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
-                        int bs, int64_t num_blocks, int* device_status, cudaStream_t stream);
+                        int bs, int64_t num_blocks, int window, int* device_status, cudaStream_t stream);
 
 // bf16, D = 128: the prompt branch with empty caches (contiguous k, v of the new tokens), same kernel.
 int launch_prompt_umma(void* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,

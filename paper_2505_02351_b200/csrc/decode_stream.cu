@@ -62,6 +62,7 @@ struct StreamParams {
     int bs;
     int partition_size;
     int max_partitions;
+    int window;             // > 0: only the last `window` keys of each sequence are attended to (balanced split only)
 };
 
 template <int D>
@@ -125,6 +126,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const int P = p.partition_size, P16 = P / kTileTok;    // tiles per full partition
+    // A sequence's stream starts at the tile that holds its first attended key (tile 0 without a window) and its
+    // partitions are counted from there.
+    auto first_tile_of = [&](int n) { return p.window > 0 ? max(0, n - p.window) / kTileTok : 0; };
+    auto tiles_of = [&](int n) { return (n + kTileTok - 1) / kTileTok - first_tile_of(n); };
     const int* __restrict__ lens = p.context_lens;         // an input of the step: not written by the preceding grid
     if (lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
@@ -135,7 +140,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     long long total = 0;
     for (int s0 = 0; s0 < p.B; s0 += 32) {
         const int n = s0 + lane < p.B ? __ldg(lens + s0 + lane) : 0;
-        int tl = (n + kTileTok - 1) / kTileTok;
+        int tl = tiles_of(n);
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) tl += __shfl_xor_sync(kFull, tl, o);
         total += tl;
@@ -161,7 +166,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         cur.s = -1;
         for (int s0 = 0; s0 < p.B && cur.s < 0; s0 += 32) {
             const int n = s0 + lane < p.B ? __ldg(lens + s0 + lane) : 0;
-            const int tl = (n + kTileTok - 1) / kTileTok, np = (n + P - 1) / P;
+            const int tl = tiles_of(n), np = (tl + P16 - 1) / P16;
             int incl_t = tl, incl_p = np;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -201,8 +206,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 ++cur.s;
                 cur.n = cur.s < p.B ? __ldg(lens + cur.s) : 0;
             } while (cur.s < p.B && cur.n == 0);
-            cur.tiles = (cur.n + kTileTok - 1) / kTileTok;
-            cur.parts = (cur.n + P - 1) / P;
+            cur.tiles = tiles_of(cur.n);
+            cur.parts = (cur.tiles + P16 - 1) / P16;
         }
     };
     if (!kBalanced && cur.jt % P16 != 0) {
@@ -228,7 +233,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     // Describes the piece under `cur` in slot (piece & 3), starts the loads of its first 32 page ids, moves `cur`
     // on.  A piece is the part of one partition that lies inside this worker's range (kBalanced) or one whole
     // partition (otherwise).  desc[2i] = {s, kvh, n, first tile in the stream}, desc[2i+1] = {tiles, row of the
-    // partial result of the group's first head}.
+    // partial result of the group's first head}; tiles are numbered from the sequence's token 0.
     int pieces = 0;               // pieces described so far
     int pages_nxt = 0;            // lane l: physical page of tile l of the piece described last
     auto describe_next = [&]() {
@@ -251,10 +256,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             obase = (cur.s * p.Hq + cur.kvh * G) * p.max_partitions + part;
         }
         if (lane == 0) {
-            desc[2 * (pieces & (kDescSlots - 1))] = make_int4(cur.s, cur.kvh, cur.n, cur.jt);
+            desc[2 * (pieces & (kDescSlots - 1))] = make_int4(cur.s, cur.kvh, cur.n, first_tile_of(cur.n) + cur.jt);
             desc[2 * (pieces & (kDescSlots - 1)) + 1] = make_int4(len, obase, 0, 0);
         }
-        const int tok = (cur.jt + lane) * kTileTok;
+        const int tok = (first_tile_of(cur.n) + cur.jt + lane) * kTileTok;
         pages_nxt = lane < len ? __ldg(p.block_tables + (size_t)cur.s * p.max_blocks + tok / p.bs) : 0;
         ++pieces;
         cur.pos += len;
@@ -398,8 +403,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             sc[1] = fmaf(sc[1], qscale, sl[1] * relA);
             sc[2] = fmaf(sc[2], qscale, sl[0] * relB);
             sc[3] = fmaf(sc[3], qscale, sl[1] * relB);
-            if (ja >= cs_n) sc[0] = sc[1] = -INFINITY;
-            if (ja + 8 >= cs_n) sc[2] = sc[3] = -INFINITY;
+            const int cs_start = p.window > 0 ? max(0, cs_n - p.window) : 0;     // first attended key
+            if (ja >= cs_n || ja < cs_start) sc[0] = sc[1] = -INFINITY;
+            if (ja + 8 >= cs_n || ja + 8 < cs_start) sc[2] = sc[3] = -INFINITY;
         }
         const float m0n = fmaxf(m0, group_max(fmaxf(sc[0], sc[2])));
         const float m1n = fmaxf(m1, group_max(fmaxf(sc[1], sc[3])));
@@ -528,7 +534,7 @@ int launch_g(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams& p
 int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                          int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                         float* partial_out, float* partial_lse, void* workspace, int max_partitions,
+                         float* partial_out, float* partial_lse, void* workspace, int max_partitions, int window,
                          int* device_status, cudaStream_t stream) {
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
@@ -562,6 +568,7 @@ int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache
     p.bs = bs;
     p.partition_size = partition_size;
     p.max_partitions = max_partitions;
+    p.window = workspace ? window : 0;
     const int G = Hq / Hkv;
     if (workspace) {
         if (D == 128) return launch_g<128, true>(mk, mv, p, G, stream);

@@ -78,6 +78,7 @@ struct UmmaParams {
     int Hq;
     int Hkv;
     int bs;
+    int window;             // > 0: token at pos sees keys pos - window < j <= pos only
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -194,17 +195,18 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 }
 
 // Pass 1 over one 32-key chunk of a row's scores: t = s*qscale + slope*(key index) + bias_c, running maxima.
-// kMasked adds the causal select (keys after `pos` count as -inf); tiles left of the diagonal skip it.
+// kMasked adds the select of the visible keys, lo < key <= pos (causal bound pos; lo = pos - window, or -1);
+// tiles strictly inside that range skip it.
 template <bool kMasked>
 __device__ __forceinline__ void chunk_max(const float (&v)[32], float qscale, float slope2, float bias_c, int key0,
-                                          int pos, float (&mx)[4]) {
+                                          int pos, int lo, float (&mx)[4]) {
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
         float t0 = fmaf(v[e], qscale, fmaf(slope2, (float)e, bias_c));
         float t1 = fmaf(v[e + 1], qscale, fmaf(slope2, (float)(e + 1), bias_c));
         if (kMasked) {
-            t0 = key0 + e <= pos ? t0 : -INFINITY;
-            t1 = key0 + e + 1 <= pos ? t1 : -INFINITY;
+            t0 = (key0 + e <= pos && key0 + e > lo) ? t0 : -INFINITY;
+            t1 = (key0 + e + 1 <= pos && key0 + e + 1 > lo) ? t1 : -INFINITY;
         }
         mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], t0, t1);
     }
@@ -213,14 +215,14 @@ __device__ __forceinline__ void chunk_max(const float (&v)[32], float qscale, fl
 // Pass 2 over one chunk: p = 2^t (the maximum is folded into bias_c), bf16 pairs for the tensor core, partial sums.
 template <bool kMasked>
 __device__ __forceinline__ void chunk_exp(const float (&v)[32], float qscale, float slope2, float bias_c, int key0,
-                                          int pos, float (&sm)[4], uint32_t (&w)[16]) {
+                                          int pos, int lo, float (&sm)[4], uint32_t (&w)[16]) {
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
         float t0 = fmaf(v[2 * e], qscale, fmaf(slope2, (float)(2 * e), bias_c));
         float t1 = fmaf(v[2 * e + 1], qscale, fmaf(slope2, (float)(2 * e + 1), bias_c));
         if (kMasked) {
-            t0 = key0 + 2 * e <= pos ? t0 : -INFINITY;
-            t1 = key0 + 2 * e + 1 <= pos ? t1 : -INFINITY;
+            t0 = (key0 + 2 * e <= pos && key0 + 2 * e > lo) ? t0 : -INFINITY;
+            t1 = (key0 + 2 * e + 1 <= pos && key0 + 2 * e + 1 > lo) ? t1 : -INFINITY;
         }
         const float p0 = ex2(t0), p1 = ex2(t1);
         sm[e & 3] += p0 + p1;
@@ -259,7 +261,12 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int n = kPaged ? p.context_lens[s] : qlen;
     const int i_last = min(qlen, (qb + 1) * TQ) - 1;        // last valid new token of this block
     const int pos_last = n - qlen + i_last;                 // its position; the block sees keys 0 .. pos_last
-    const int ntiles = pos_last / kTN + 1;
+    // Tiles tile_lo .. tile_hi hold the keys the block sees: up to pos_last, and with a local window no further
+    // back than window - 1 keys before the block's first token.
+    const int tile_hi = pos_last / kTN;
+    const int pos_first = n - qlen + qb * TQ;
+    const int tile_lo = p.window > 0 ? max(0, pos_first - p.window + 1) / kTN : 0;
+    const int ntiles = tile_hi - tile_lo + 1;
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
@@ -299,15 +306,15 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         const int32_t* table = kPaged ? p.block_tables + (size_t)s * p.max_blocks : nullptr;
         const int sub = lane & 7;                           // lanes 0-7 fetch one 16-token slice each
-        auto page_of = [&](int j) -> int {         // j counts processed tiles; the tile is ntiles - 1 - j
-            const int tok = (ntiles - 1 - j) * kTN + sub * kSub;
+        auto page_of = [&](int j) -> int {         // j counts processed tiles; the tile is tile_hi - j
+            const int tok = (tile_hi - j) * kTN + sub * kSub;
             return (kPaged && lane < 8 && tok < n) ? __ldg(table + tok / p.bs) : -1;
         };
         int page = page_of(0);
         for (int j = 0; j < ntiles; ++j) {
             const int st = j % kKvStages;
             const int page_next = j + 1 < ntiles ? page_of(j + 1) : -1;
-            const int j0 = (ntiles - 1 - j) * kTN;
+            const int j0 = (tile_hi - j) * kTN;
             const int nsub = min(kTN / kSub, (n - j0 + kSub - 1) / kSub);     // slices that hold cached tokens
             const int tok = j0 + sub * kSub;
             const int row = (page * p.Hkv + kvh) * p.bs + tok % p.bs;          // row of the [rows, D] view
@@ -390,6 +397,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const bool valid = i < qlen;
         // Rows past the end of the block are computed as copies of the last valid position and never stored.
         const int pos = n - qlen + min(i, i_last);
+        const int lo = p.window > 0 ? pos - p.window : -1;       // keys lo < j <= pos are visible
         const int h = kvh * G + hg;
         const float qscale = p.scale * kLog2e;
         const float slope2 = p.slopes ? p.slopes[h] * kLog2e : 0.f;
@@ -399,7 +407,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         bool ok = true;
 
         for (int j = 0; j < ntiles; ++j) {
-            const int sb = j & 1, j0 = (ntiles - 1 - j) * kTN;
+            const int sb = j & 1, j0 = (tile_hi - j) * kTN;
             ok = __all_sync(kFull, mbar_wait(&s_full[sb], (j >> 1) & 1, p.status));
             if (!ok) break;
             tc_fence_after();
@@ -408,8 +416,9 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // ---- pass 1: the row's scores for the tile's 128 keys (Eq. 3), only their maximum is kept.  The
             // loops over the four 32-key chunks are not unrolled: with one warp per scheduler the code has to
             // stay inside the instruction cache.
-            // Only tiles on the diagonal need the causal select; the choice is made per warp.
-            const bool masked = __any_sync(kFull, j0 + kTN - 1 > pos);
+            // Only tiles on the diagonal (and at the far edge of a local window) need the select; the choice is
+            // made per warp.
+            const bool masked = __any_sync(kFull, j0 + kTN - 1 > pos || j0 <= lo);
             const float bias0 = fmaf(slope2, (float)j0, c_row);       // ALiBi term of the tile's first key
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
@@ -417,8 +426,8 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 float v[32];
                 tmem_ld32(s_addr + c * 32, v);
                 const float bias_c = fmaf(slope2, (float)(c * 32), bias0);
-                if (masked) chunk_max<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, mx);
-                else chunk_max<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, mx);
+                if (masked) chunk_max<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, mx);
+                else chunk_max<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, mx);
             }
             const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 
@@ -457,8 +466,8 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 uint32_t w[16];
                 tmem_ld32(s_addr + c * 32, v);
                 const float bias_c = fmaf(slope2, (float)(c * 32), bias_m);
-                if (masked) chunk_exp<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, sm, w);
-                else chunk_exp<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, sm, w);
+                if (masked) chunk_exp<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, sm, w);
+                else chunk_exp<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, sm, w);
                 tmem_st16(s_addr + c * 16, w);
             }
             const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
@@ -577,7 +586,7 @@ int launch_g(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv
 int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens, int max_q_len,
                         const void* k_cache, const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
-                        int bs, int64_t num_blocks, int* device_status, cudaStream_t stream) {
+                        int bs, int64_t num_blocks, int window, int* device_status, cudaStream_t stream) {
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull || total_q_tokens <= 0) return OPT_GQA_ERR_SHAPE;
     if (B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
@@ -598,6 +607,7 @@ int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, in
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.bs = bs;
+    p.window = window;
     return launch_g<true>(mq, mk, mv, p, B, G, max_q_len, stream);
 }
 
@@ -623,6 +633,7 @@ int launch_prompt_umma(void* out, const void* q, const void* k, const void* v, c
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.bs = 16;
+    p.window = 0;
     return launch_g<false>(mq, mk, mv, p, B, G, max_q_len, stream);
 }
 

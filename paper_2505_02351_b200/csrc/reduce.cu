@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(kBalWarps * 32)
 reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_out,
                        const float* __restrict__ partial_lse, const long long* __restrict__ header,
                        const long long* __restrict__ seq_info, const int32_t* __restrict__ context_lens, int rows,
-                       int Hq, int Hkv, int partition_size) {
+                       int Hq, int Hkv, int partition_size, int window) {
     constexpr int V = D / 32;             // columns per lane
     constexpr int RPB = kBalWarps / WPR;  // rows per CTA
     __shared__ float s_num[kBalWarps][D];
@@ -102,7 +102,10 @@ reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_ou
     const bool active = row < rows;
     const int s = active ? row / Hq : 0, h = active ? row % Hq : 0, G = Hq / Hkv, kvh = h / G, hh = h % G;
     const int n = active ? context_lens[s] : 0;             // an input of the step, not produced by the decode grid
-    const int np = (n + partition_size - 1) / partition_size;
+    // the sequence's stream starts at the tile of its first attended key; partitions are counted from there
+    const int P16 = partition_size / 16;
+    const int tiles = (n + 15) / 16 - (window > 0 ? max(0, n - window) / 16 : 0);
+    const int np = (tiles + P16 - 1) / P16;
     grid_dependency_wait();                                 // the pieces come from the decode grid
 
     int R = 0;
@@ -110,7 +113,6 @@ reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_ou
     const float* po = partial_out;
     if (np > 0) {
         const long long total = header[0], workers = header[1];
-        const int tiles = (n + 15) / 16;
         const long long first_tile = seq_info[2 * s] * Hkv + (long long)kvh * tiles;
         const long long first_part = seq_info[2 * s + 1] * Hkv + (long long)kvh * np;
         // worker whose range [floor(T w / W), floor(T (w + 1) / W)) holds tile x: floor(((x + 1) W - 1) / T)
@@ -202,38 +204,38 @@ int launch_reduce(void* out, const float* partial_out, const float* partial_lse,
 
 template <typename T, int D, int WPR>
 static int launch_reduce_balanced_w(void* out, const char* ws, const BalancedLayout& L, const int32_t* context_lens,
-                                    int B, int Hq, int Hkv, int partition_size, cudaStream_t stream) {
+                                    int B, int Hq, int Hkv, int partition_size, int window, cudaStream_t stream) {
     const int rows = B * Hq, rpb = kBalWarps / WPR;
     return launch_dependent(reduce_balanced_kernel<T, D, WPR>, dim3((unsigned)((rows + rpb - 1) / rpb)),
                             dim3(kBalWarps * 32), 0, stream, static_cast<T*>(out),
                             reinterpret_cast<const float*>(ws + L.out), reinterpret_cast<const float*>(ws + L.lse),
                             reinterpret_cast<const long long*>(ws + L.header),
                             reinterpret_cast<const long long*>(ws + L.seq_info), context_lens, rows, Hq, Hkv,
-                            partition_size);
+                            partition_size, window);
 }
 
 template <typename T, int D>
 static int launch_reduce_balanced_t(void* out, const char* ws, const BalancedLayout& L, const int32_t* context_lens,
-                                    int B, int Hq, int Hkv, int partition_size, cudaStream_t stream) {
+                                    int B, int Hq, int Hkv, int partition_size, int window, cudaStream_t stream) {
     // About 8192 warps in all: 8 per row for a few long rows, 1 per row for batches of many rows.
     const long long rows = (long long)B * Hq;
-    if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
-    if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
-    if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
-    return launch_reduce_balanced_w<T, D, 1>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+    if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    return launch_reduce_balanced_w<T, D, 1>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
 }
 
 int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
-                           int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream) {
+                           int D, int partition_size, int max_partitions, int window, int dtype, cudaStream_t stream) {
     const BalancedLayout L = balanced_layout(B, Hq, Hkv, D, max_partitions);
     const char* ws = static_cast<const char*>(workspace);
     if (dtype == OPT_GQA_BF16) {
         if (D == 128)
-            return launch_reduce_balanced_t<__nv_bfloat16, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
-        return launch_reduce_balanced_t<__nv_bfloat16, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+            return launch_reduce_balanced_t<__nv_bfloat16, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+        return launch_reduce_balanced_t<__nv_bfloat16, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
     }
-    if (D == 128) return launch_reduce_balanced_t<float, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
-    return launch_reduce_balanced_t<float, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, stream);
+    if (D == 128) return launch_reduce_balanced_t<float, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    return launch_reduce_balanced_t<float, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
 }
 
 }  // namespace optgqa
