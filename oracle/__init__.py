@@ -42,6 +42,7 @@ def lib() -> ctypes.CDLL:
         _lib.oracle_partition_partials.restype = ctypes.c_int
         _lib.oracle_reduce.restype = ctypes.c_int
         _lib.oracle_prompt_attention.restype = ctypes.c_int
+        _lib.oracle_qkv_project_int4.restype = ctypes.c_int
         _lib.oracle_alibi_slopes.restype = None
         _lib.oracle_unpage.restype = None
     return _lib
@@ -182,3 +183,19 @@ def unpage(cache, table, n: int, kvh: int, dtype: str) -> np.ndarray:
     lib().oracle_unpage(_p(dst), _p(cache), _p(table), ctypes.c_int(n), ctypes.c_int(kvh),
                         ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(bs), ctypes.c_int(DTYPES[dtype]))
     return dst
+
+
+def qkv_project_int4(x, qweight, scales, qzeros, gs: int) -> np.ndarray:
+    """y [T, N] = x [T, K] (bf16 bits) times the 4-bit group-quantised W [K, N] (Eq. 1, weights of Q, K, V side by side)."""
+    x, scales = _check_store(x, "bf16"), _check_store(scales, "bf16")
+    qweight = np.ascontiguousarray(qweight, dtype=np.uint32)
+    qzeros = np.ascontiguousarray(qzeros, dtype=np.uint32)
+    T, K = x.shape
+    N = qweight.shape[1]
+    assert qweight.shape == (K // 8, N) and scales.shape == (K // gs, N) and qzeros.shape == (K // gs, N // 8)
+    y = np.zeros((T, N), dtype=np.float64)
+    rc = lib().oracle_qkv_project_int4(_p(y), _p(x), _p(qweight), _p(scales), _p(qzeros), ctypes.c_int(T),
+                                       ctypes.c_int(K), ctypes.c_int(N), ctypes.c_int(gs))
+    if rc != 0:
+        raise ValueError("bad shapes")
+    return y

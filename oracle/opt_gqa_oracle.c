@@ -286,3 +286,36 @@ int oracle_prompt_attention(double* out, const void* q, const void* k, const voi
     }
     return 0;
 }
+
+/*
+ * Q/K/V projection of Eq. 1 (Q = X W_Q, K = X W_K, V = X W_V) with the three weight matrices stored
+ * side by side as one 4-bit group-quantised matrix W [K, N], N = (Hq + 2 Hkv) D.  The paper names GPTQ
+ * in its title but states no storage format; the reading taken here is the common group-wise one:
+ *
+ *   qweight [K/8, N]   uint32   code of row 8r+i, column n in bits 4i..4i+3 of word (r, n)
+ *   scales  [K/gs, N]  bf16     one scale per group of gs consecutive rows and column
+ *   qzeros  [K/gs, N/8] uint32  zero point of group g, column 8c+i in bits 4i..4i+3 of word (g, c)
+ *   w[k][n] = scales[k/gs][n] * (code[k][n] - zero[k/gs][n])
+ *   y[t][n] = sum_k x[t][k] * w[k][n]        x [T, K] bf16, y [T, N] double
+ *
+ * Columns 0 .. Hq D - 1 of y are the token's query, the next Hkv D its key, the last Hkv D its value.
+ */
+int oracle_qkv_project_int4(double* y, const void* x, const uint32_t* qweight, const void* scales,
+                            const uint32_t* qzeros, int T, int K, int N, int gs) {
+    if (T < 0 || K <= 0 || N <= 0 || gs <= 0 || K % 8 != 0 || N % 8 != 0 || K % gs != 0) return -1;
+    #pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) {
+                int g = k / gs;
+                int code = (int)((qweight[(int64_t)(k / 8) * N + n] >> (4 * (k % 8))) & 0xFu);
+                int zero = (int)((qzeros[(int64_t)g * (N / 8) + n / 8] >> (4 * (n % 8))) & 0xFu);
+                double w = load_elem(scales, (int64_t)g * N + n, 1) * (double)(code - zero);
+                acc += load_elem(x, (int64_t)t * K + k, 1) * w;
+            }
+            y[(int64_t)t * N + n] = acc;
+        }
+    }
+    return 0;
+}

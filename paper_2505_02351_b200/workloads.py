@@ -200,3 +200,37 @@ def make_config(cfg: int, poison: bool = False, shrink: int = 1, seed_offset: in
         5: dict(dtype="bf16", Hq=32, Hkv=8, D=128, bs=16, partition_size=0),
     }[cfg]
     return make_custom(CONFIG_NAMES[cfg], context_lens=n, q_lens=ql, seed=seed, poison=poison, **shape)
+
+
+@dataclass
+class Int4Projection:
+    """Inputs of the 4-bit Q/K/V projection: activations and one group-quantised weight matrix [K, N]."""
+    x: torch.Tensor        # [T, K] bf16
+    qweight: torch.Tensor  # [K/8, N] int32, eight 4-bit codes of consecutive rows per word
+    scales: torch.Tensor   # [K/gs, N] bf16
+    qzeros: torch.Tensor   # [K/gs, N/8] int32, eight 4-bit zero points of consecutive columns per word
+    gs: int
+
+    @property
+    def K(self) -> int:
+        return self.x.shape[1]
+
+    @property
+    def N(self) -> int:
+        return self.qweight.shape[1]
+
+    def weight_bytes(self) -> int:
+        """Bytes of codes, scales and zero points in the interchange layout (read once per projection)."""
+        return self.qweight.numel() * 4 + self.scales.numel() * 2 + self.qzeros.numel() * 4
+
+
+def make_int4_projection(seed: int, T: int, K: int, N: int, gs: int = 128) -> Int4Projection:
+    """Random codes and zero points (uniform words), scales near 0.008 (the step of a 4-bit grid over
+    weights of standard deviation ~0.02), activations N(0,1) rounded to bf16."""
+    rng = np.random.default_rng(seed)
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    qweight = torch.from_numpy(rng.integers(0, 2**32, size=(K // 8, N), dtype=np.uint32).view(np.int32))
+    qzeros = torch.from_numpy(rng.integers(0, 2**32, size=(K // gs, N // 8), dtype=np.uint32).view(np.int32))
+    scales = (0.006 + 0.004 * torch.rand((K // gs, N), generator=gen, dtype=torch.float32)).to(torch.bfloat16)
+    x = torch.randn((T, K), generator=gen, dtype=torch.float32).to(torch.bfloat16)
+    return Int4Projection(x=x, qweight=qweight, scales=scales, qzeros=qzeros, gs=gs)

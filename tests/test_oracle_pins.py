@@ -403,3 +403,54 @@ def test_prompt_attention_is_prefill_over_a_cache_holding_only_the_new_tokens():
     # the first token of every sequence sees only itself
     for s in range(3):
         assert np.allclose(got[qsl[s]], brute.widen(v)[qsl[s]].repeat(4, axis=0), atol=1e-15)
+
+
+# ---- 4-bit Q/K/V projection (Eq. 1 with group-quantised weights) ----
+
+def _bf16_bits(a):
+    return W.storage_numpy(torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16))
+
+
+def test_int4_projection_hand_example():
+    """One 8 x 8 block typed by hand: row k of every column holds code k except row 0, which holds the
+    column index; zero point of column i is 7 - i; every scale is 0.5."""
+    qweight = np.array([[0x76543210 + n for n in range(8)]], dtype=np.uint32)
+    qzeros = np.array([[0x01234567]], dtype=np.uint32)
+    scales = _bf16_bits(np.full((1, 8), 0.5))
+    e0 = _bf16_bits(np.eye(8)[0:1])
+    e3 = _bf16_bits(np.eye(8)[3:4])
+    y0 = oracle.qkv_project_int4(e0, qweight, scales, qzeros, 8)
+    y3 = oracle.qkv_project_int4(e3, qweight, scales, qzeros, 8)
+    assert y0.tolist() == [[-3.5, -2.5, -1.5, -0.5, 0.5, 1.5, 2.5, 3.5]]
+    assert y3.tolist() == [[-2.0, -1.5, -1.0, -0.5, 0.0, 0.5, 1.0, 1.5]]
+
+
+def test_int4_projection_is_an_integer_matmul_when_scales_are_powers_of_two():
+    rng = np.random.default_rng(5)
+    T, K, N, gs = 3, 64, 24, 16
+    qweight = rng.integers(0, 2**32, size=(K // 8, N), dtype=np.uint32)
+    qzeros = rng.integers(0, 2**32, size=(K // gs, N // 8), dtype=np.uint32)
+    exps = rng.integers(-2, 3, size=(K // gs, N))
+    xi = rng.integers(-8, 9, size=(T, K))
+    codes = np.stack([(qweight >> np.uint32(4 * i)) & np.uint32(15) for i in range(8)], axis=1).reshape(K, N).astype(np.int64)
+    zeros = np.stack([(qzeros >> np.uint32(4 * i)) & np.uint32(15) for i in range(8)], axis=2).reshape(K // gs, N).astype(np.int64)
+    want = np.zeros((T, N))
+    for g in range(K // gs):
+        want += (xi[:, g * gs:(g + 1) * gs] @ (codes[g * gs:(g + 1) * gs] - zeros[g])) * np.exp2(exps[g])
+    got = oracle.qkv_project_int4(_bf16_bits(xi), qweight, _bf16_bits(np.exp2(exps)), qzeros, gs)
+    assert np.array_equal(got, want)
+
+
+def test_int4_projection_group_whose_codes_equal_its_zero_points_contributes_nothing():
+    p = W.make_int4_projection(9, 2, 64, 16, gs=32)
+    qweight = p.qweight.numpy().view(np.uint32).copy()
+    qzeros = p.qzeros.numpy().view(np.uint32)
+    zeros = np.stack([(qzeros >> np.uint32(4 * i)) & np.uint32(15) for i in range(8)], axis=2).reshape(2, 16)
+    qweight[4:8] = (zeros[1] * np.uint32(0x11111111))[None, :]          # rows 32..63 = group 1
+    x = W.storage_numpy(p.x)
+    s = W.storage_numpy(p.scales)
+    y = oracle.qkv_project_int4(x, qweight, s, qzeros, 32)
+    x2 = x.copy()
+    x2[:, 32:] = _bf16_bits(np.full((2, 32), 3.0))
+    assert np.array_equal(y, oracle.qkv_project_int4(x2, qweight, s, qzeros, 32))
+    assert np.abs(y).max() > 0
