@@ -273,6 +273,42 @@ int opt_gqa_prompt_attention(void* out, const void* q, const void* k, const void
                              int Hkv, int D, int dtype, void* stream);
 
 /*
+ * Q/K/V projection of Eq. 1 (Q = X W_Q, K = X W_K, V = X W_V) for the T tokens of a decode step, from
+ * 4-bit group-quantised weights, with the keys and values written where the rest of the step reads them:
+ * Algorithm 1, "Reshape and store K, V into C_K, C_V".  The paper names GPTQ in its title and gives no
+ * storage format; the interchange layout taken here is the common group-wise one, W [K, N] with the
+ * three matrices side by side (columns 0 .. Hq D - 1 query, then Hkv D key, then Hkv D value):
+ *
+ *   qweight  [K/8, N]    uint32   code of row 8r+i, column n in bits 4i .. 4i+3 of word (r, n)
+ *   scales   [K/gs, N]   bf16
+ *   qzeros   [K/gs, N/8] uint32   zero point of group g, column 8c+i in bits 4i .. 4i+3 of word (g, c)
+ *   w[k][n] = scales[k/gs][n] * (code[k][n] - zero[k/gs][n]),   y[t][n] = sum_k x[t][k] w[k][n]
+ *
+ * opt_gqa_int4_prepack rewrites these three arrays once into the layout the kernel streams (`packed`,
+ * opt_gqa_int4_packed_bytes(K, N, gs) bytes of device memory, 16-byte aligned; all four DEVICE pointers).
+ * K a multiple of gs, gs 64 or 128, N a multiple of 32.  opt_gqa_int4_packed_bytes returns 0 otherwise.
+ *
+ * opt_gqa_qkv_project_int4: x [T, K] bf16 (K = the model width), N = (Hq + 2 Hkv) D.
+ *   q_out          [T, Hq, D]  bf16, always written
+ *   k_out, v_out   [T, Hkv, D] bf16, or both NULL
+ *   k_cache, v_cache           the paged pool [num_blocks, Hkv, bs, D] bf16, or both NULL; token t's key and
+ *                              value go to slot_mapping[t] exactly as in opt_gqa_cache_append (a negative
+ *                              slot, or one past the pool, skips the token)
+ * At least one of the two destinations for K/V must be given.  Sums are accumulated in fp32 and rounded
+ * once to bf16.  The kernel is sized for the few tokens of a decode step (up to 16 per pass over the
+ * weights); larger T is accepted and takes one pass per 16 tokens.  All pointers are DEVICE pointers,
+ * 16-byte aligned.  Errors as everywhere in this header; nothing is launched on an error.
+ */
+size_t opt_gqa_int4_packed_bytes(int K, int N, int gs);
+
+int opt_gqa_int4_prepack(void* packed, const uint32_t* qweight, const void* scales, const uint32_t* qzeros, int K,
+                         int N, int gs, void* stream);
+
+int opt_gqa_qkv_project_int4(void* q_out, void* k_out, void* v_out, void* k_cache, void* v_cache,
+                             const int64_t* slot_mapping, const void* x, const void* packed, int T, int K, int Hq,
+                             int Hkv, int D, int bs, int64_t num_blocks, int gs, void* stream);
+
+/*
  * One decode step of the attention layer, Algorithm 2 from "Store reshaped K, V
  * into C_K, C_V" to "Compute context attention with caches": cache_append of the
  * B new tokens (k_new, v_new [B, Hkv, D], slot_mapping [B]), then decode, then --

@@ -24,6 +24,9 @@ _c = ctypes
 _vp, _i, _i64, _f = _c.c_void_p, _c.c_int, _c.c_int64, _c.c_float
 
 SIGNATURES = {
+    "opt_gqa_int4_packed_bytes": (ctypes.c_size_t, [_i, _i, _i]),
+    "opt_gqa_int4_prepack": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "opt_gqa_qkv_project_int4": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i64, _i, _vp]),
     "opt_gqa_cache_append": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i64, _i, _vp]),
     "opt_gqa_paged_attention_decode": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                             _i, _vp, _vp, _i, _i, _vp]),
@@ -243,6 +246,30 @@ def prompt_attention(out, q, k, v, q_start_loc, max_q_len: int, alibi_slopes, sc
     _check(load().opt_gqa_prompt_attention(
         _ptr(out), _ptr(q), _ptr(k), _ptr(v), _ptr(q_start_loc), T, max_q_len, _ptr(alibi_slopes), scale, B, Hq, Hkv,
         D, _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_prompt_attention")
+
+
+def int4_packed_bytes(K: int, N: int, gs: int) -> int:
+    return int(load().opt_gqa_int4_packed_bytes(K, N, gs))
+
+
+def int4_prepack(packed, qweight, scales, qzeros, gs: int, stream=None) -> None:
+    """Rewrite qweight [K/8, N] int32, scales [K/gs, N] bf16, qzeros [K/gs, N/8] int32 into the kernel's layout."""
+    K, N = qweight.shape[0] * 8, qweight.shape[1]
+    assert scales.dtype == torch.bfloat16 and qweight.dtype == torch.int32 and qzeros.dtype == torch.int32
+    assert packed.numel() * packed.element_size() >= int4_packed_bytes(K, N, gs) > 0
+    _check(load().opt_gqa_int4_prepack(_ptr(packed), _ptr(qweight), _ptr(scales), _ptr(qzeros), K, N, gs,
+                                       _stream(stream)), "opt_gqa_int4_prepack")
+
+
+def qkv_project_int4(q_out, x, packed, Hq: int, Hkv: int, D: int, gs: int, k_out=None, v_out=None, k_cache=None,
+                     v_cache=None, slot_mapping=None, stream=None) -> None:
+    """q, k, v = x W (Eq. 1) from 4-bit weights; k, v go to k_out/v_out and/or into the paged cache."""
+    T, K = x.shape
+    assert x.dtype == torch.bfloat16 and q_out.dtype == torch.bfloat16
+    num_blocks, bs = (k_cache.shape[0], k_cache.shape[2]) if k_cache is not None else (0, 0)
+    _check(load().opt_gqa_qkv_project_int4(
+        _ptr(q_out), _ptr(k_out), _ptr(v_out), _ptr(k_cache), _ptr(v_cache), _ptr(slot_mapping), _ptr(x),
+        _ptr(packed), T, K, Hq, Hkv, D, bs, num_blocks, gs, _stream(stream)), "opt_gqa_qkv_project_int4")
 
 
 def step_staging_bytes(B: int, Hq: int, Hkv: int, D: int, max_blocks_per_seq: int, dtype: torch.dtype) -> int:

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libopt_gqa.so")
-SOURCES = ["api.cu", "cache_append.cu", "decode.cu", "decode_tc.cu", "decode_stream.cu", "reduce.cu", "prefill.cu", "prefill_umma.cu", "no_alloc.cu"]
+SOURCES = ["api.cu", "cache_append.cu", "decode.cu", "decode_tc.cu", "decode_stream.cu", "reduce.cu", "prefill.cu", "prefill_umma.cu", "no_alloc.cu", "qkv_int4.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
