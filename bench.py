@@ -303,6 +303,70 @@ def prefill_report(dev, steps: int, warmup: int) -> dict:
             "flop_per_launch": pb.flops(), "bound": "tensor"}
 
 
+def projection_report(dev) -> dict:
+    """Side measurement of the 4-bit Q/K/V projection that precedes the step: one launch per layer-sized weight
+    matrix, rotating through enough distinct matrices to exceed L2.  The launches are shorter than a foreign call
+    from Python, so they are timed as one captured graph."""
+    import time
+
+    import torch
+    from paper_2505_02351_b200 import binding
+    from paper_2505_02351_b200 import workloads as W
+
+    lib = binding.load()
+    peak, kind = measured_peak()
+    out = {}
+    side = torch.cuda.Stream()
+    for name, T, K, Hq, Hkv, D in (("width4096_32q4kv_T8", 8, 4096, 32, 4, 128), ("width8192_64q8kv_T8", 8, 8192, 64, 8, 128),
+                                   ("width8192_64q8kv_T16", 16, 8192, 64, 8, 128)):
+        N, gs = (Hq + 2 * Hkv) * D, 128
+        p = W.make_int4_projection(11, T, K, N, gs)
+        nbytes = binding.int4_packed_bytes(K, N, gs)
+        copies = max(2, -(-300_000_000 // nbytes))
+        packed = torch.empty((copies, nbytes), dtype=torch.uint8, device=dev)
+        binding.int4_prepack(packed[0], p.qweight.to(dev), p.scales.to(dev), p.qzeros.to(dev), gs)
+        for i in range(1, copies):
+            packed[i].copy_(packed[0])
+        x = p.x.to(dev)
+        q = torch.empty((T, Hq, D), dtype=torch.bfloat16, device=dev)
+        k = torch.empty((T, Hkv, D), dtype=torch.bfloat16, device=dev)
+        v = torch.empty_like(k)
+        calls = [(q.data_ptr(), k.data_ptr(), v.data_ptr(), None, None, None, x.data_ptr(), packed[i].data_ptr(), T, K,
+                  Hq, Hkv, D, 0, 0, gs, side.cuda_stream) for i in range(copies)]
+        f = lib.opt_gqa_qkv_project_int4
+        with torch.cuda.stream(side):
+            for i in range(copies):
+                check(f(*calls[i]), "qkv_project_int4")
+        side.synchronize()
+        per_graph = copies * max(1, 120 // copies)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(per_graph):
+                check(f(*calls[i % copies]), "qkv_project_int4")
+        t_end = time.time() + 0.3                      # replays first: clocks up, caches in steady state
+        while time.time() < t_end:
+            for _ in range(20):
+                graph.replay()
+            torch.cuda.synchronize()
+        spans = []
+        for _ in range(20):
+            start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            start.record()
+            graph.replay()
+            end.record()
+            torch.cuda.synchronize()
+            spans.append(start.elapsed_time(end))
+        us = sorted(spans)[len(spans) // 2] * 1e3 / per_graph
+        alg = p.weight_bytes() + x.numel() * 2 + T * N * 2
+        out[name] = {"us_per_launch": us, "GBs": alg / (us * 1e-6) / 1e9, "frac_of_peak": alg / (us * 1e-6) / 1e9 / peak,
+                     "algorithmic_bytes_per_launch": alg, "weight_copies_rotated": copies, "bound": "hbm",
+                     "timing": f"median over 20 replays of a graph of {per_graph} launches, CUDA events around each replay",
+                     "peak_kind": f"of {kind}"}
+        del packed, graph
+        torch.cuda.empty_cache()
+    return out
+
+
 def check(rc: int, what: str):
     if rc != 0:
         raise RuntimeError(f"{what} failed with status {rc}")
@@ -540,6 +604,8 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the short side measurements of the other workloads")
     ap.add_argument("--prefill-only", action="store_true",
                     help="run only the chunked-prefill side measurement and print its report (profiling runs)")
+    ap.add_argument("--projection-only", action="store_true",
+                    help="run only the 4-bit Q/K/V projection side measurement and print its report (profiling runs)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
 
@@ -568,6 +634,10 @@ def main():
     if args.prefill_only:
         if rank == 0:
             print(json.dumps(prefill_report(dev, args.steps or 20, max(3, args.warmup or 3))), flush=True)
+        return
+    if args.projection_only:
+        if rank == 0:
+            print(json.dumps(projection_report(dev)), flush=True)
         return
     steps = args.steps if args.steps is not None else 4000
     warmup = max(3, args.warmup if args.warmup is not None else 50)
@@ -643,6 +713,7 @@ def main():
             del b2, w2
             torch.cuda.empty_cache()
         extra[W.CONFIG_NAMES[5]] = prefill_report(dev, 20, 3)
+        extra["int4_qkv_projection"] = projection_report(dev)
         line["other_workloads"] = extra
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
