@@ -29,7 +29,7 @@
 namespace optgqa {
 namespace {
 
-constexpr int kProjWarps = 16;        // warps of a CTA; they split K between them
+constexpr int kProjWarps = 8;         // warps of a CTA; they split K between them
 constexpr int kFeatPerCta = 32;       // output features of a CTA: two m16 tiles
 constexpr int kRedStride = 36;        // floats between the tokens' rows of the cross-warp sum (bank spread)
 
@@ -64,7 +64,7 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
 
 // NT: token tiles of eight per CTA; CPG: 64-row chunks per quantisation group.
 template <int NT, int CPG>
-__global__ void __launch_bounds__(kProjWarps * 32, 1) qkv_int4_kernel(const ProjParams p) {
+__global__ void __launch_bounds__(kProjWarps * 32, 2) qkv_int4_kernel(const ProjParams p) {
     constexpr int PF = NT == 1 ? 4 : 2;   // chunks in flight per warp; a multiple of CPG
     static_assert(PF % CPG == 0, "ring must hold whole groups");
     constexpr int GSLOTS = PF / CPG;
@@ -94,18 +94,20 @@ __global__ void __launch_bounds__(kProjWarps * 32, 1) qkv_int4_kernel(const Proj
     uint4 W[PF][2];
     uint4 X[PF][NT][2];
     uint32_t SZ[GSLOTS][4];
-    auto fetch = [&](int u, int kc) {
+    auto fetch_w = [&](int u, int kc) {
         W[u][0] = __ldcs(w0 + (size_t)kc * 32);
         W[u][1] = __ldcs(w1 + (size_t)kc * 32);
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            X[u][nt][0] = __ldg(xrow[nt] + kc * 8);
-            X[u][nt][1] = __ldg(xrow[nt] + kc * 8 + 4);
-        }
         if (u % CPG == 0) {
             const uint32_t* s = szcol + (size_t)(kc / CPG) * p.N;
 #pragma unroll
             for (int i = 0; i < 4; ++i) SZ[u / CPG][i] = __ldg(s + 8 * i);
+        }
+    };
+    auto fetch_x = [&](int u, int kc) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            X[u][nt][0] = __ldcg(xrow[nt] + kc * 8);
+            X[u][nt][1] = __ldcg(xrow[nt] + kc * 8 + 4);
         }
     };
 
@@ -117,9 +119,15 @@ __global__ void __launch_bounds__(kProjWarps * 32, 1) qkv_int4_kernel(const Proj
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[m][nt][i] = 0.f;
 
+    // the first weights are requested before the preceding kernel of the stream has finished: they do not
+    // depend on it, only the activations do
 #pragma unroll
     for (int u = 0; u < PF; ++u)
-        if (kc0 + u < kc1) fetch(u, kc0 + u);
+        if (kc0 + u < kc1) fetch_w(u, kc0 + u);
+    grid_dependency_wait();
+#pragma unroll
+    for (int u = 0; u < PF; ++u)
+        if (kc0 + u < kc1) fetch_x(u, kc0 + u);
 
     uint32_t zpair[4];
     float scale[4];
@@ -159,7 +167,10 @@ __global__ void __launch_bounds__(kProjWarps * 32, 1) qkv_int4_kernel(const Proj
                     }
                 }
             }
-            if (kc + u + PF < kc1) fetch(u, kc + u + PF);
+            if (kc + u + PF < kc1) {
+                fetch_w(u, kc + u + PF);
+                fetch_x(u, kc + u + PF);
+            }
             if (u % CPG == CPG - 1) {
 #pragma unroll
                 for (int m = 0; m < 2; ++m)
@@ -183,6 +194,7 @@ __global__ void __launch_bounds__(kProjWarps * 32, 1) qkv_int4_kernel(const Proj
     __syncthreads();
 
     // one thread per (token, pair of features): 16 pairs x 8 NT tokens
+    static_assert(16 * 8 * NT <= kProjWarps * 32, "the epilogue needs a thread per output pair");
     if (threadIdx.x < 16 * 8 * NT) {
         const int tl = threadIdx.x >> 4, f = (threadIdx.x & 15) * 2;
         const int t = t0 + tl;
@@ -322,12 +334,9 @@ extern "C" int opt_gqa_qkv_project_int4(void* q_out, void* k_out, void* v_out, v
     const long long chunks = ((long long)T + 8 * NT - 1) / (8 * NT);
     if (chunks > 65535) return OPT_GQA_ERR_SHAPE;
     dim3 grid((unsigned)(Nl / kFeatPerCta), (unsigned)chunks), block(kProjWarps * 32);
-    if (NT == 1) {
-        if (gs == 64) qkv_int4_kernel<1, 1><<<grid, block, 0, cs>>>(p);
-        else qkv_int4_kernel<1, 2><<<grid, block, 0, cs>>>(p);
-    } else {
-        if (gs == 64) qkv_int4_kernel<2, 1><<<grid, block, 0, cs>>>(p);
-        else qkv_int4_kernel<2, 2><<<grid, block, 0, cs>>>(p);
-    }
-    return cudaGetLastError() == cudaSuccess ? OPT_GQA_OK : OPT_GQA_ERR_CUDA;
+    if (NT == 1)
+        return gs == 64 ? launch_dependent(qkv_int4_kernel<1, 1>, grid, block, 0, cs, p)
+                        : launch_dependent(qkv_int4_kernel<1, 2>, grid, block, 0, cs, p);
+    return gs == 64 ? launch_dependent(qkv_int4_kernel<2, 1>, grid, block, 0, cs, p)
+                    : launch_dependent(qkv_int4_kernel<2, 2>, grid, block, 0, cs, p);
 }
