@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 DEFAULT_PARTITION = {2: 256, 3: 512, 4: 512}
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised
 # under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {3: 378_694_400 + 8_636_160}   # profiles/decode_stream_cfg3.md
+NCU_TRAFFIC_BYTES = {3: 378_697_984 + 8_272_128}   # profiles/decode_stream_cfg3.md
 
 
 # ----------------------------------------------------------------------------- distributed plumbing
@@ -303,7 +303,11 @@ def prefill_report(dev, steps: int, warmup: int) -> dict:
             "flop_per_launch": pb.flops(), "bound": "tensor"}
 
 
-def projection_report(dev) -> dict:
+PROJECTION_SHAPES = (("width4096_32q4kv_T8", 8, 4096, 32, 4, 128), ("width8192_64q8kv_T8", 8, 8192, 64, 8, 128),
+                     ("width8192_64q8kv_T16", 16, 8192, 64, 8, 128))
+
+
+def projection_report(dev, only=None) -> dict:
     """Side measurement of the 4-bit Q/K/V projection that precedes the step: one launch per layer-sized weight
     matrix, rotating through enough distinct matrices to exceed L2.  The launches are shorter than a foreign call
     from Python, so they are timed as one captured graph."""
@@ -317,8 +321,9 @@ def projection_report(dev) -> dict:
     peak, kind = measured_peak()
     out = {}
     side = torch.cuda.Stream()
-    for name, T, K, Hq, Hkv, D in (("width4096_32q4kv_T8", 8, 4096, 32, 4, 128), ("width8192_64q8kv_T8", 8, 8192, 64, 8, 128),
-                                   ("width8192_64q8kv_T16", 16, 8192, 64, 8, 128)):
+    for name, T, K, Hq, Hkv, D in PROJECTION_SHAPES:
+        if only is not None and name != only:
+            continue
         N, gs = (Hq + 2 * Hkv) * D, 128
         p = W.make_int4_projection(11, T, K, N, gs)
         nbytes = binding.int4_packed_bytes(K, N, gs)
@@ -606,6 +611,8 @@ def main():
                     help="run only the chunked-prefill side measurement and print its report (profiling runs)")
     ap.add_argument("--projection-only", action="store_true",
                     help="run only the 4-bit Q/K/V projection side measurement and print its report (profiling runs)")
+    ap.add_argument("--projection-shape", default=None, choices=[s[0] for s in PROJECTION_SHAPES],
+                    help="with --projection-only: measure this shape alone")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
 
@@ -637,7 +644,7 @@ def main():
         return
     if args.projection_only:
         if rank == 0:
-            print(json.dumps(projection_report(dev)), flush=True)
+            print(json.dumps(projection_report(dev, args.projection_shape)), flush=True)
         return
     steps = args.steps if args.steps is not None else 4000
     warmup = max(3, args.warmup if args.warmup is not None else 50)
