@@ -208,7 +208,9 @@ static int prefill_checked(bool allow_umma, int window, void* out, const void* q
     if (!aligned16(out) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
-    if (allow_umma && D == 128)
+    // the tcgen05 kernel folds scale into its score tile and needs it positive; anything else takes the other kernel
+    if (window > 0 && !(scale > 0.f)) return OPT_GQA_ERR_SHAPE;
+    if (allow_umma && D == 128 && scale > 0.f)
         return launch_prefill_umma(out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
                                    max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, bs, num_blocks,
                                    window, status, static_cast<cudaStream_t>(stream));
@@ -254,7 +256,8 @@ int opt_gqa_prompt_attention(void* out, const void* q, const void* k, const void
                              int Hkv, int D, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
-    if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, 16) || D != 128) return OPT_GQA_ERR_SHAPE;
+    if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, 16) || D != 128 || !(scale > 0.f))
+        return OPT_GQA_ERR_SHAPE;
     if (B == 0 || max_q_len == 0 || total_q_tokens == 0) return OPT_GQA_OK;
     if (!out || !q || !k || !v || !q_start_loc) return OPT_GQA_ERR_NULL;
     if (!aligned16(out) || !aligned16(q) || !aligned16(k) || !aligned16(v)) return OPT_GQA_ERR_ALIGN;

@@ -55,7 +55,16 @@ constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kOffQ = 0;
 constexpr int kOffK = kQBytes;
 constexpr int kOffV = kOffK + kKvStages * kTileBytes;
-constexpr int kOffBar = kOffV + kKvStages * kTileBytes;
+// The ALiBi term rides on the tensor core as one more k-step of S = Q K^T: an extension of Q that holds
+// slope_h / scale split over three bf16 values, against an extension of K that holds the key's index inside
+// the tile three times.  Both are 16-dim K-major operands without swizzle: 8-row x 16-byte core matrices of
+// 128 contiguous bytes, the two 8-dim halves of a row group 128 bytes apart, row groups 256 bytes apart.
+constexpr int kExtRowGroupBytes = 256;
+constexpr int kQxBytes = kRows / 8 * kExtRowGroupBytes;   // 4 KiB
+constexpr int kKpBytes = kTN / 8 * kExtRowGroupBytes;     // 2 KiB
+constexpr int kOffQx = kOffV + kKvStages * kTileBytes;
+constexpr int kOffKp = kOffQx + kQxBytes;
+constexpr int kOffBar = kOffKp + kKpBytes;
 // barriers: q_full, k_full[3], k_empty[3], v_full[3], v_empty[3], s_full[2], p_full[2]; then the TMEM base word
 constexpr int kNumBars = 1 + 4 * kKvStages + 4;
 constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;   // + slack to align the tiles to 1 KiB
@@ -95,6 +104,13 @@ __device__ __forceinline__ void tc_commit(uint64_t* bar) {
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
            (1ull << 46) | (2ull << 61);
+}
+
+// Shared-memory matrix descriptor without swizzle (core matrices of 8 rows x 16 bytes): lbo = distance between the
+// core matrices of one row group along K, sbo = distance between row groups.
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46);
 }
 
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128, N = n, A K-major, B K-major or MN-major.
@@ -194,32 +210,32 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// Pass 1 over one 32-key chunk of a row's scores: t = s*qscale + slope*(key index) + bias_c, running maxima.
-// kMasked adds the select of the visible keys, lo < key <= pos (causal bound pos; lo = pos - window, or -1);
-// tiles strictly inside that range skip it.
+// Pass 1 over one 32-key chunk of a row's raw scores s = q.k + (slope/scale)*(key index in the tile): running
+// maxima.  The map to log2 units, t = s*qscale + (tile constant), is increasing, so it is applied to the maximum
+// afterwards.  kMasked adds the select of the visible keys, lo < key <= pos (causal bound pos; lo = pos - window,
+// or -1); tiles strictly inside that range skip it.
 template <bool kMasked>
-__device__ __forceinline__ void chunk_max(const float (&v)[32], float qscale, float slope2, float bias_c, int key0,
-                                          int pos, int lo, float (&mx)[4]) {
+__device__ __forceinline__ void chunk_max(const float (&v)[32], int key0, int pos, int lo, float (&mx)[4]) {
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
-        float t0 = fmaf(v[e], qscale, fmaf(slope2, (float)e, bias_c));
-        float t1 = fmaf(v[e + 1], qscale, fmaf(slope2, (float)(e + 1), bias_c));
+        float s0 = v[e], s1 = v[e + 1];
         if (kMasked) {
-            t0 = (key0 + e <= pos && key0 + e > lo) ? t0 : -INFINITY;
-            t1 = (key0 + e + 1 <= pos && key0 + e + 1 > lo) ? t1 : -INFINITY;
+            s0 = (key0 + e <= pos && key0 + e > lo) ? s0 : -INFINITY;
+            s1 = (key0 + e + 1 <= pos && key0 + e + 1 > lo) ? s1 : -INFINITY;
         }
-        mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], t0, t1);
+        mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], s0, s1);
     }
 }
 
-// Pass 2 over one chunk: p = 2^t (the maximum is folded into bias_c), bf16 pairs for the tensor core, partial sums.
+// Pass 2 over one chunk: p = 2^(s*qscale + bias) with the tile's ALiBi constant and the row maximum folded into
+// bias; bf16 pairs for the tensor core, partial sums.
 template <bool kMasked>
-__device__ __forceinline__ void chunk_exp(const float (&v)[32], float qscale, float slope2, float bias_c, int key0,
-                                          int pos, int lo, float (&sm)[4], uint32_t (&w)[16]) {
+__device__ __forceinline__ void chunk_exp(const float (&v)[32], float qscale, float bias, int key0, int pos, int lo,
+                                          float (&sm)[4], uint32_t (&w)[16]) {
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
-        float t0 = fmaf(v[2 * e], qscale, fmaf(slope2, (float)(2 * e), bias_c));
-        float t1 = fmaf(v[2 * e + 1], qscale, fmaf(slope2, (float)(2 * e + 1), bias_c));
+        float t0 = fmaf(v[2 * e], qscale, bias);
+        float t1 = fmaf(v[2 * e + 1], qscale, bias);
         if (kMasked) {
             t0 = (key0 + 2 * e <= pos && key0 + 2 * e > lo) ? t0 : -INFINITY;
             t1 = (key0 + 2 * e + 1 <= pos && key0 + 2 * e + 1 > lo) ? t1 : -INFINITY;
@@ -284,6 +300,30 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         tmem_slot[1] = 0;       // set by mbar_wait's callers when a wait gave up (see the end of the kernel)
         fence_barrier_init();
+    }
+    // Extension operands of the ALiBi k-step (see kOffQx): row r of Q's holds slope_h / scale as a sum of three
+    // bf16 values, row e of K's the index e three times; dims 3..15 are zero.
+    const bool alibi = p.slopes != nullptr;
+    if (alibi) {
+        if (threadIdx.x < kRows) {
+            const int r = threadIdx.x;
+            const float a = p.slopes[kvh * G + r % G] / p.scale;
+            const __nv_bfloat16 a0 = __float2bfloat16_rn(a);
+            const __nv_bfloat16 a1 = __float2bfloat16_rn(a - __bfloat162float(a0));
+            const __nv_bfloat16 a2 = __float2bfloat16_rn(a - __bfloat162float(a0) - __bfloat162float(a1));
+            char* row = smem + kOffQx + (r >> 3) * kExtRowGroupBytes + (r & 7) * 16;
+            *reinterpret_cast<uint4*>(row) = make_uint4((uint32_t)__bfloat16_as_ushort(a0) | ((uint32_t)__bfloat16_as_ushort(a1) << 16),
+                                                        (uint32_t)__bfloat16_as_ushort(a2), 0u, 0u);
+            *reinterpret_cast<uint4*>(row + 128) = make_uint4(0u, 0u, 0u, 0u);
+        } else {
+            for (int e = threadIdx.x - kRows; e < kTN; e += kThreads - kRows) {
+                const uint32_t eb = __bfloat16_as_ushort(__float2bfloat16_rn((float)e));      // exact: e < 256
+                char* row = smem + kOffKp + (e >> 3) * kExtRowGroupBytes + (e & 7) * 16;
+                *reinterpret_cast<uint4*>(row) = make_uint4(eb | (eb << 16), eb, 0u, 0u);
+                *reinterpret_cast<uint4*>(row + 128) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        fence_proxy_async();
     }
     if (warp == 5) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -383,6 +423,9 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                             smem_desc(q_addr + (ks >> 2) * kQHalfBytes + (ks & 3) * 32, 16, 1024),
                             smem_desc(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024), idesc_s, ks > 0);
                 }
+                if (alibi)
+                    umma_ss(tmem_base + kColS + sb * kTN, smem_desc_plain(smem_u32(smem + kOffQx), 128, kExtRowGroupBytes),
+                            smem_desc_plain(smem_u32(smem + kOffKp), 128, kExtRowGroupBytes), idesc_s, true);
                 tc_commit(&s_full[sb]);
                 tc_commit(&k_empty[st]);
                 if (j >= 1) ok = issue_pv(j - 1);
@@ -425,11 +468,11 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             for (int c = 0; c < kTN / 32; ++c) {
                 float v[32];
                 tmem_ld32(s_addr + c * 32, v);
-                const float bias_c = fmaf(slope2, (float)(c * 32), bias0);
-                if (masked) chunk_max<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, mx);
-                else chunk_max<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, mx);
+                if (masked) chunk_max<true>(v, j0 + c * 32, pos, lo, mx);
+                else chunk_max<false>(v, j0 + c * 32, pos, lo, mx);
             }
-            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            // qscale > 0: the largest raw score gives the largest t (and -inf stays -inf)
+            const float m_tile = fmaf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), qscale, bias0);
 
             // ---- running maximum: move it (and rescale l and O) only when it grew by more than the threshold
             // (true for the first tile in which the row sees a key: m_used = -inf until then)
@@ -465,9 +508,8 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 float v[32];
                 uint32_t w[16];
                 tmem_ld32(s_addr + c * 32, v);
-                const float bias_c = fmaf(slope2, (float)(c * 32), bias_m);
-                if (masked) chunk_exp<true>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, sm, w);
-                else chunk_exp<false>(v, qscale, slope2, bias_c, j0 + c * 32, pos, lo, sm, w);
+                if (masked) chunk_exp<true>(v, qscale, bias_m, j0 + c * 32, pos, lo, sm, w);
+                else chunk_exp<false>(v, qscale, bias_m, j0 + c * 32, pos, lo, sm, w);
                 tmem_st16(s_addr + c * 16, w);
             }
             const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
