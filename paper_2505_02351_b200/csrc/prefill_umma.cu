@@ -227,23 +227,96 @@ __device__ __forceinline__ void chunk_max(const float (&v)[32], int key0, int po
     }
 }
 
+// Two fp32 values in one 64-bit register, for the packed fp32 instructions of sm_100 (one issue slot for two lanes).
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+#ifndef OPT_GQA_PF_POLY_PERIOD
+#define OPT_GQA_PF_POLY_PERIOD 0
+#endif
+// Every kPolyPeriod-th pair of a chunk takes 2^t from the FMA pipe instead of the special-function unit (0: none).
+constexpr int kPolyPeriod = OPT_GQA_PF_POLY_PERIOD;
+
+// 2^t for two values without the special-function unit: t = n + f with n = round(t) (taken from the low mantissa
+// bits of t + 1.5 * 2^23), 2^f on [-1/2, 1/2] by a cubic whose relative error (8e-5) is far below the bf16
+// rounding that follows, and n added to the exponent field.  t is clamped at -126: 2^-126 stands in for
+// anything smaller, masked keys included.
+__device__ __forceinline__ uint64_t exp2_pair_fma(uint64_t t2) {
+    float t0, t1;
+    unpack_f2(t2, t0, t1);
+    t2 = pack_f2(fmaxf(t0, -126.f), fmaxf(t1, -126.f));
+    const uint64_t magic = pack_f2(12582912.f, 12582912.f), neg_magic = pack_f2(-12582912.f, -12582912.f);
+    const uint64_t y2 = add2(t2, magic);
+    const uint64_t n2 = add2(y2, neg_magic);
+    const uint64_t f2 = fma2(n2, pack_f2(-1.f, -1.f), t2);
+    uint64_t r2 = fma2(pack_f2(0.05508868f, 0.05508868f), f2, pack_f2(0.24260405f, 0.24260405f));
+    r2 = fma2(r2, f2, pack_f2(0.69327623f, 0.69327623f));
+    r2 = fma2(r2, f2, pack_f2(0.99992895f, 0.99992895f));
+    float y0, y1, r0, r1;
+    unpack_f2(y2, y0, y1);
+    unpack_f2(r2, r0, r1);
+    return pack_f2(__int_as_float(__float_as_int(r0) + (__float_as_int(y0) << 23)),
+                   __int_as_float(__float_as_int(r1) + (__float_as_int(y1) << 23)));
+}
+
 // Pass 2 over one chunk: p = 2^(s*qscale + bias) with the tile's ALiBi constant and the row maximum folded into
-// bias; bf16 pairs for the tensor core, partial sums.
+// bias; bf16 pairs for the tensor core; returns the chunk's sum of p.
 template <bool kMasked>
-__device__ __forceinline__ void chunk_exp(const float (&v)[32], float qscale, float bias, int key0, int pos, int lo,
-                                          float (&sm)[4], uint32_t (&w)[16]) {
+__device__ __forceinline__ float chunk_exp(const float (&v)[32], float qscale, float bias, int key0, int pos, int lo,
+                                           uint32_t (&w)[16]) {
+    if (kMasked) {
+        float sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-        float t0 = fmaf(v[2 * e], qscale, bias);
-        float t1 = fmaf(v[2 * e + 1], qscale, bias);
-        if (kMasked) {
+        for (int e = 0; e < 16; ++e) {
+            float t0 = fmaf(v[2 * e], qscale, bias);
+            float t1 = fmaf(v[2 * e + 1], qscale, bias);
             t0 = (key0 + 2 * e <= pos && key0 + 2 * e > lo) ? t0 : -INFINITY;
             t1 = (key0 + 2 * e + 1 <= pos && key0 + 2 * e + 1 > lo) ? t1 : -INFINITY;
+            const float p0 = ex2(t0), p1 = ex2(t1);
+            sm[e & 3] += p0 + p1;
+            w[e] = pack2(p0, p1);
         }
-        const float p0 = ex2(t0), p1 = ex2(t1);
-        sm[e & 3] += p0 + p1;
+        return (sm[0] + sm[1]) + (sm[2] + sm[3]);
+    }
+    const uint64_t qs2 = pack_f2(qscale, qscale), b2 = pack_f2(bias, bias);
+    uint64_t sm2[2] = {pack_f2(0.f, 0.f), pack_f2(0.f, 0.f)};
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        const uint64_t t2 = fma2(pack_f2(v[2 * e], v[2 * e + 1]), qs2, b2);
+        uint64_t p2;
+        float p0, p1;
+        if (kPolyPeriod > 0 && e % kPolyPeriod == kPolyPeriod - 1) {
+            p2 = exp2_pair_fma(t2);
+            unpack_f2(p2, p0, p1);
+        } else {
+            float t0, t1;
+            unpack_f2(t2, t0, t1);
+            p0 = ex2(t0);
+            p1 = ex2(t1);
+            p2 = pack_f2(p0, p1);
+        }
+        sm2[e & 1] = add2(sm2[e & 1], p2);
         w[e] = pack2(p0, p1);
     }
+    float s0, s1;
+    unpack_f2(add2(sm2[0], sm2[1]), s0, s1);
+    return s0 + s1;
 }
 
 // kPaged: K/V come from the paged cache through block_tables (2-D maps over [rows, D]); otherwise from contiguous
@@ -502,17 +575,16 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // (a row that has not seen a key yet has only -inf scores: subtract 0 so that they give p = 0)
             const float m_sub = m_used == -INFINITY ? 0.f : m_used;
             const float bias_m = bias0 - m_sub;
-            float sm[4] = {0.f, 0.f, 0.f, 0.f};
+            float sum = 0.f;
 #pragma unroll 1
             for (int c = 0; c < kTN / 32; ++c) {
                 float v[32];
                 uint32_t w[16];
                 tmem_ld32(s_addr + c * 32, v);
-                if (masked) chunk_exp<true>(v, qscale, bias_m, j0 + c * 32, pos, lo, sm, w);
-                else chunk_exp<false>(v, qscale, bias_m, j0 + c * 32, pos, lo, sm, w);
+                if (masked) sum += chunk_exp<true>(v, qscale, bias_m, j0 + c * 32, pos, lo, w);
+                else sum += chunk_exp<false>(v, qscale, bias_m, j0 + c * 32, pos, lo, w);
                 tmem_st16(s_addr + c * 16, w);
             }
-            const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
             l += sum;
 
             if (j0 + kTN > n) {
