@@ -208,7 +208,8 @@ int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q, const void
  *   q_start_loc   [B+1] int32              prefix sums of q_len_s, device memory
  *   total_q_tokens HOST value: rows of q and out (= q_start_loc[B]); rows are read up to it
  *   max_q_len     HOST value >= max_s q_len_s (sizes the grid)
- * D = 128 runs on tcgen05.mma with accumulators in tensor memory; D = 64 on warp-level mma.
+ * D = 128 with scale > 0 runs on tcgen05.mma with accumulators in tensor memory; D = 64, or a
+ * scale that is not positive, on warp-level mma.
  */
 int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
                                     int max_q_len, const void* k_cache, const void* v_cache,
@@ -238,7 +239,7 @@ int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t*
  * opt_gqa_paged_attention_decode_local: the balanced split and its merge in one call (arguments as
  * opt_gqa_paged_attention_decode_balanced followed by opt_gqa_paged_attention_reduce_balanced; out
  * [B, Hq, D] is written; bf16 caches, partition_size > 0).  opt_gqa_paged_attention_prefill_local:
- * arguments as opt_gqa_paged_attention_prefill (bf16, D = 128).  window > 0 is required.
+ * arguments as opt_gqa_paged_attention_prefill (bf16, D = 128, scale > 0).  window > 0 is required.
  */
 int opt_gqa_paged_attention_decode_local(void* out, const void* q, const void* k_cache, const void* v_cache,
                                          const int32_t* block_tables, int max_blocks_per_seq,

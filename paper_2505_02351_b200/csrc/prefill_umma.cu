@@ -5,11 +5,12 @@
 // One CTA per (query block, KV head, sequence).  The G query heads of the group times TQ = 128 / G
 // consecutive new tokens are the 128 rows of the CTA's tiles, so every K/V tile is fetched once for
 // the whole group ("Shared Key-Value").  Six warps, three roles:
-//   warps 0-3  one thread per row: read the 128 x kTN score tile S from tensor memory, add the ALiBi
-//              term slope_h*(j - pos) and mask j > pos from the indices (Eq. 3), keep the row's
-//              running maximum and denominator (Eq. 4, online; two passes over S, first the maximum,
-//              then p), write p as bf16 back into tensor memory over S, rescale O when the maximum
-//              moved, and store the normalised rows
+//   warps 0-3  one thread per row: read the row of the 128 x kTN score tile S from tensor memory (it
+//              already holds the ALiBi term slope_h*(j - j0) of Eq. 3 relative to the tile's first
+//              key j0; the rest of the term is a constant of the row and tile), mask j > pos from the
+//              indices, keep the row's running maximum and denominator (Eq. 4, online; two passes
+//              over the scores in registers, first the maximum, then p), write p as bf16 back into
+//              tensor memory over S, rescale O when the maximum moved, and store the normalised rows
 //   warp 4     producer: walks the block table and fetches kTN-key K and V tiles (2-D TMA boxes of
 //              16 token rows x 128 bytes, 128-byte swizzle) into a ring, plus the Q tile
 //   warp 5     one thread issues S = Q K^T (operands in shared memory) and O += P V (P from tensor
@@ -18,10 +19,11 @@
 // j-1's P V while the row threads do tile j's softmax.  Tiles are taken from the diagonal backwards
 // (nearest keys first): the ALiBi term falls with distance, so a row's maximum is set by the first
 // tiles it sees and O is rescaled only when the maximum still grows by more than 2^8 -- in forward
-// order the bias alone would move it every tile.  The softmax is bound by instruction issue (exp2 on
-// the special-function unit, max on the half-rate pipe) with one row warp per scheduler, so the
-// default shape is 64-key tiles in a two-stage ring: two CTAs fit on an SM (96 KiB of shared memory
-// and 256 tensor-memory columns each) and one CTA's exp2 phase overlaps the other's maximum phase.
+// order the bias alone would move it every tile.  The ALiBi term inside a tile is added by the tensor core
+// itself (a ninth k-step, see kOffQx), so a row thread spends one max per two scores in the first pass and one
+// packed FMA, two exp2, one packed add and one conversion per two scores in the second.  The default shape is
+// 64-key tiles in a two-stage ring: two CTAs fit on an SM (102 KiB of shared memory and 256 tensor-memory
+// columns each) and one CTA's row warps run while the other's wait.
 // Every wait is a bounded mbarrier wait.
 #include "tma_mma.cuh"
 
@@ -536,13 +538,26 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // made per warp.
             const bool masked = __any_sync(kFull, j0 + kTN - 1 > pos || j0 <= lo);
             const float bias0 = fmaf(slope2, (float)j0, c_row);       // ALiBi term of the tile's first key
+            // the whole row of the tile is read once (both loads in flight together) and kept in registers for
+            // both passes
+            float v[kTN / 32][32];
+            {
+                uint32_t raw[kTN / 32][32];
+#pragma unroll
+                for (int c = 0; c < kTN / 32; ++c) tmem_ld32_issue(s_addr + c * 32, raw[c]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < kTN / 32; ++c) {
+                    tmem_pin(raw[c]);
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[c][e] = __uint_as_float(raw[c][e]);
+                }
+            }
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
+#pragma unroll
             for (int c = 0; c < kTN / 32; ++c) {
-                float v[32];
-                tmem_ld32(s_addr + c * 32, v);
-                if (masked) chunk_max<true>(v, j0 + c * 32, pos, lo, mx);
-                else chunk_max<false>(v, j0 + c * 32, pos, lo, mx);
+                if (masked) chunk_max<true>(v[c], j0 + c * 32, pos, lo, mx);
+                else chunk_max<false>(v[c], j0 + c * 32, pos, lo, mx);
             }
             // qscale > 0: the largest raw score gives the largest t (and -inf stays -inf)
             const float m_tile = fmaf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), qscale, bias0);
@@ -576,13 +591,11 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const float m_sub = m_used == -INFINITY ? 0.f : m_used;
             const float bias_m = bias0 - m_sub;
             float sum = 0.f;
-#pragma unroll 1
+#pragma unroll
             for (int c = 0; c < kTN / 32; ++c) {
-                float v[32];
                 uint32_t w[16];
-                tmem_ld32(s_addr + c * 32, v);
-                if (masked) sum += chunk_exp<true>(v, qscale, bias_m, j0 + c * 32, pos, lo, w);
-                else sum += chunk_exp<false>(v, qscale, bias_m, j0 + c * 32, pos, lo, w);
+                if (masked) sum += chunk_exp<true>(v[c], qscale, bias_m, j0 + c * 32, pos, lo, w);
+                else sum += chunk_exp<false>(v[c], qscale, bias_m, j0 + c * 32, pos, lo, w);
                 tmem_st16(s_addr + c * 16, w);
             }
             l += sum;
