@@ -71,6 +71,23 @@ def test_prefill_with_one_new_token_is_the_decode_result():
     assert np.max(np.abs(got - dec)) <= TOL
 
 
+@pytest.mark.parametrize("scale", [0.0, -0.05, 0.5])
+def test_scales_that_are_not_the_usual_one(scale):
+    """The tcgen05 kernel needs a positive scale (it takes the row maximum before scaling); zero and negative
+    scales are routed to the other kernel.  Either way the result is the oracle's."""
+    wl = W.make_custom("pfs", "bf16", 8, 2, 128, 16, [300, 70], q_lens=[130, 70], seed=37)
+    wl.scale = scale
+    _check(wl)
+
+
+def test_steep_and_flat_slopes_on_the_tensor_core_bias():
+    """slope / scale is split over three bf16 values inside the kernel: check slopes far from the usual ones."""
+    for mult in (0.0, 1e-3, 7.0):
+        wl = W.make_custom("pfb", "bf16", 8, 2, 128, 16, [700, 129], q_lens=[200, 129], seed=38)
+        wl.alibi_slopes = wl.alibi_slopes * mult
+        _check(wl)
+
+
 def test_empty_sequences_and_no_new_tokens():
     # a sequence that contributes no new tokens leaves no row; the others are unaffected
     wl = W.make_custom("pf0", "bf16", 4, 2, 128, 16, [50, 64, 20], q_lens=[0, 64, 20], seed=32, poison=True)
