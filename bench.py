@@ -401,6 +401,15 @@ def _step_fns(batch: DeviceBatch, stream):
                 step=lambda i: check(f_step(*a_step[i % R]), "decode_step"))
 
 
+def step_launches(batch: DeviceBatch) -> int:
+    """Kernels one opt_gqa_decode_step call launches: decode + reduce on the split path, plus the separate append
+    unless the decode kernel stores the new tokens itself (bf16 split with at most 1024 (sequence, KV head) streams)."""
+    if batch.P == 0:
+        return 2
+    fused = batch.balanced and batch.wl.B * batch.wl.Hkv <= 1024
+    return 2 if fused else 3
+
+
 def run_timed(batch: DeviceBatch, steps: int, warmup: int):
     """Warm-up, then `steps` steps timed with CUDA events on the launching stream.
 
@@ -423,7 +432,7 @@ def run_timed(batch: DeviceBatch, steps: int, warmup: int):
     end.record(stream)
     torch.cuda.synchronize()
     barrier()
-    return start.elapsed_time(end), steps * (3 if f["split"] else 2)
+    return start.elapsed_time(end), steps * step_launches(batch)
 
 
 def run_kernel_timing(batch: DeviceBatch, steps: int, warmup: int):
@@ -451,7 +460,7 @@ def run_kernel_timing(batch: DeviceBatch, steps: int, warmup: int):
     for i in range(steps):
         if i not in evs:
             f["step"](warmup + i)
-            launches += 3 if f["split"] else 2
+            launches += step_launches(batch)
             continue
         nb = DECODE_BATCH if (i // EVENT_EVERY) % 2 == 0 else 1
         f["append"](warmup + i)
@@ -693,7 +702,7 @@ def main():
         "config": {"workload": wl.name, "batch_per_gpu": wl.B, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.D,
                    "block_size": wl.bs, "storage_dtype": wl.dtype, "partition_size": P,
                    "context_tokens_per_gpu": int(wl.context_lens.sum()), "parallelism": f"dp{world} (by sequence, no collective)",
-                   "step": "cache_append + decode + reduce",
+                   "step": "opt_gqa_decode_step: append of one token per sequence (stored by the decode kernel) + decode + reduce",
                    "l2": f"{args.copies} distinct KV pool copies ({pool_bytes / 1e9:.2f} GB) rotated between steps; "
                          f"each step reads {wl.kv_bytes() / 1e6:.0f} MB (> 126 MB L2)"},
         "hbm_tbs_step": alg * tokens_all / wl.B / (total_ms / steps * 1e-3) / 1e12,

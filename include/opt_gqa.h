@@ -319,6 +319,10 @@ int opt_gqa_qkv_project_int4(void* q_out, void* k_out, void* v_out, void* k_cach
  * the balanced split (decode_balanced + reduce_balanced), fp32 caches one partial
  * per partition (partial_out followed by partial_lse at the start of workspace).
  * Other arguments as in the calls it chains.  out [B, Hq, D] is always written.
+ * On the bf16 split path with at most 1024 (sequence, KV head) streams no separate append kernel
+ * runs: the decode kernel stores sequence s's new token to slot_mapping[s] itself, just before it
+ * fetches the tile that holds position context_lens[s] - 1 (a sequence with context_lens 0 has no
+ * such tile and stores nothing).
  */
 int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,
                         const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,

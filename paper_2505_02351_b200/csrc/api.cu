@@ -127,7 +127,7 @@ static int decode_balanced_checked(const void* q, const void* k_cache, const voi
                                    const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
                                    int64_t num_blocks, int partition_size, void* workspace, int max_partitions,
-                                   int window, int dtype, void* stream) {
+                                   int window, int dtype, void* stream, const FusedAppend* append = nullptr) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0 || partition_size <= 0 ||
@@ -142,7 +142,7 @@ static int decode_balanced_checked(const void* q, const void* k_cache, const voi
     if (!status) return OPT_GQA_ERR_CUDA;
     return launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
                                 scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, nullptr, nullptr, workspace,
-                                max_partitions, window, status, static_cast<cudaStream_t>(stream));
+                                max_partitions, window, status, static_cast<cudaStream_t>(stream), append);
 }
 
 int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, const void* v_cache,
@@ -267,6 +267,9 @@ int opt_gqa_prompt_attention(void* out, const void* q, const void* k, const void
                               status, static_cast<cudaStream_t>(stream));
 }
 
+// Streams (sequence x KV head) up to which opt_gqa_decode_step lets the streaming kernel store the new tokens.
+static constexpr long long kFusedAppendMaxStreams = 1024;
+
 int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,
                         const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,
                         int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,
@@ -274,17 +277,33 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
                         int partition_size, void* workspace, int max_partitions, int dtype, void* stream) {
     if (!out) return B == 0 ? OPT_GQA_OK : OPT_GQA_ERR_NULL;
     if (partition_size > 0 && !workspace && B > 0) return OPT_GQA_ERR_NULL;
-    int rc = opt_gqa_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, B, Hkv, D, bs, num_blocks, dtype,
-                                  stream);
-    if (rc != OPT_GQA_OK) return rc;
+    int rc;
     if (dtype == OPT_GQA_BF16 && partition_size > 0 && B > 0) {
-        rc = opt_gqa_paged_attention_decode_balanced(q, k_cache, v_cache, block_tables, max_blocks_per_seq,
-                                                     context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks,
-                                                     partition_size, workspace, max_partitions, dtype, stream);
+        // bf16 split.  With few (sequence, KV head) streams the streaming kernel stores the new tokens itself, each
+        // just before the tile that holds it is fetched, and the separate launch is saved; with thousands of
+        // streams those stores would stall the workers more often than the launch costs.
+        const bool fuse = (long long)B * Hkv <= kFusedAppendMaxStreams;
+        if (fuse) {
+            // the argument checks of the slot-mapped write
+            if (Hkv <= 0 || (D != 64 && D != 128) || (bs != 16 && bs != 32) || num_blocks <= 0) return OPT_GQA_ERR_SHAPE;
+            if (!k_new || !v_new || !k_cache || !v_cache || !slot_mapping) return OPT_GQA_ERR_NULL;
+            if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache))
+                return OPT_GQA_ERR_ALIGN;
+        } else {
+            rc = opt_gqa_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, B, Hkv, D, bs, num_blocks, dtype,
+                                      stream);
+            if (rc != OPT_GQA_OK) return rc;
+        }
+        const FusedAppend fa = {k_new, v_new, k_cache, v_cache, slot_mapping};
+        rc = decode_balanced_checked(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
+                                     scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, max_partitions, 0,
+                                     dtype, stream, fuse ? &fa : nullptr);
         if (rc != OPT_GQA_OK) return rc;
         return opt_gqa_paged_attention_reduce_balanced(out, workspace, context_lens, B, Hq, Hkv, D, partition_size,
                                                        max_partitions, dtype, stream);
     }
+    rc = opt_gqa_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, B, Hkv, D, bs, num_blocks, dtype, stream);
+    if (rc != OPT_GQA_OK) return rc;
     float* partial_out = static_cast<float*>(workspace);
     float* partial_lse =
         partial_out ? partial_out + (size_t)(B > 0 ? B : 0) * Hq * (max_partitions > 0 ? max_partitions : 0) * D

@@ -186,13 +186,25 @@ inline BalancedLayout balanced_layout(int B, int Hq, int Hkv, int D, int max_par
     return L;
 }
 
+// The step's new K/V rows for the streaming kernel to store itself (Algorithm 2, "Store reshaped K, V into C_K,
+// C_V"): the worker that is about to fetch the tile holding a sequence's last position first writes that sequence's
+// new token to its slot, which saves the separate launch of the slot-mapped write.
+struct FusedAppend {
+    const void* k_new;              // [B, Hkv, D] bf16
+    const void* v_new;
+    void* k_cache;
+    void* v_cache;
+    const int64_t* slot_mapping;    // [B]; negative: nothing to store
+};
+
 // bf16, partition_size > 0: persistent streaming kernel, one worker per warp (decode_stream.cu).
 // workspace == nullptr writes one partial per partition to partial_out / partial_lse; otherwise the balanced split.
+// append != nullptr (balanced split only): see FusedAppend.
 int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                          int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
                          float* partial_out, float* partial_lse, void* workspace, int max_partitions, int window,
-                         int* device_status, cudaStream_t stream);
+                         int* device_status, cudaStream_t stream, const FusedAppend* append = nullptr);
 
 // Merge of the balanced split's pieces (reduce.cu).
 int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,

@@ -14,6 +14,12 @@
 // still being consumed.  The cut is computed by every warp from context_lens alone
 // (two coalesced passes), so there is no scheduler state in global memory.
 //
+// When the caller hands over the step's new K/V rows (Algorithm 2, "Store reshaped K, V into C_K, C_V"), the
+// worker that is about to fetch the tile holding a sequence's last position stores that sequence's new token
+// to its slot first -- plain stores, a generic-to-async proxy fence, then the bulk copy -- so the step needs no
+// separate launch for the slot-mapped write.  Every tile belongs to exactly one worker, so nobody else reads
+// the row before it is there.
+//
 // Per tile the warp computes, transposed so that the 16 tokens are the rows and the
 // (up to 8) heads of the group the columns of an m16n8k16 tile,
 //   S^T = K q^T              8 k-steps over the head dimension          (Eq. 3, dot products)
@@ -63,6 +69,12 @@ struct StreamParams {
     int partition_size;
     int max_partitions;
     int window;             // > 0: only the last `window` keys of each sequence are attended to (balanced split only)
+    // fused store of the step's new tokens (all null when the cache already holds them)
+    const uint4* k_new;
+    const uint4* v_new;
+    uint4* k_cache_w;
+    uint4* v_cache_w;
+    const int64_t* slot_mapping;
 };
 
 template <int D>
@@ -269,7 +281,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     };
 
     // ------------------------------------------------------------------ issue side
-    int is_piece = -1, is_j = 0, is_ntile = 0, is_kvh = 0, is_tile0 = 0, is_s = 0;
+    int is_piece = -1, is_j = 0, is_ntile = 0, is_kvh = 0, is_tile0 = 0, is_s = 0, is_last_tile = -1;
     int pages_cur = 0;
     uint32_t issued = 0, consumed = 0;     // tiles over the worker's whole stream: ring slot = count % kStages
     int cs_piece = -1;
@@ -289,6 +301,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             is_s = d0.x;
             is_kvh = d0.y;
             is_tile0 = d0.w;
+            is_last_tile = (d0.z - 1) / kTileTok;          // the tile that holds the sequence's newest token
             const uint32_t* qh = reinterpret_cast<const uint32_t*>(
                 p.q + ((size_t)d0.x * p.Hq + (size_t)d0.y * G + (g < G ? g : 0)) * D);
 #pragma unroll
@@ -304,6 +317,24 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             // pieces longer than 512 tokens: the next 32 page ids
             const int tok = (is_tile0 + is_j + lane) * kTileTok;
             pages_cur = is_j + lane < is_ntile ? __ldg(p.block_tables + (size_t)is_s * p.max_blocks + tok / p.bs) : 0;
+        }
+        if (p.k_new && is_tile0 + is_j == is_last_tile) {
+            // The step's new token of this sequence lies in the tile about to be fetched: store its K and V rows
+            // of this head first (as the slot-mapped write would), and order the stores before the bulk copy.
+            const long long slot = __ldg(p.slot_mapping + is_s);
+            if (slot >= 0) {
+                constexpr int VEC = D * 2 / 16;                  // 16-byte vectors per row
+                if (lane < 2 * VEC) {
+                    const bool is_v = lane >= VEC;
+                    const int vi = lane % VEC;
+                    const size_t src = ((size_t)is_s * p.Hkv + is_kvh) * VEC + vi;
+                    const size_t dst = (((size_t)(slot / p.bs) * p.Hkv + is_kvh) * p.bs + (size_t)(slot % p.bs)) * VEC + vi;
+                    if (is_v) p.v_cache_w[dst] = __ldg(p.v_new + src);
+                    else p.k_cache_w[dst] = __ldg(p.k_new + src);
+                }
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+            }
+            __syncwarp();
         }
         const int phys = __shfl_sync(kFull, pages_cur, is_j & 31);
         if (lane == 0) {
@@ -535,7 +566,7 @@ int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                          int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
                          float* partial_out, float* partial_lse, void* workspace, int max_partitions, int window,
-                         int* device_status, cudaStream_t stream) {
+                         int* device_status, cudaStream_t stream, const FusedAppend* append) {
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
     CUtensorMap mk, mv;
@@ -569,6 +600,12 @@ int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache
     p.partition_size = partition_size;
     p.max_partitions = max_partitions;
     p.window = workspace ? window : 0;
+    const bool fuse = workspace && append;
+    p.k_new = fuse ? static_cast<const uint4*>(append->k_new) : nullptr;
+    p.v_new = fuse ? static_cast<const uint4*>(append->v_new) : nullptr;
+    p.k_cache_w = fuse ? static_cast<uint4*>(append->k_cache) : nullptr;
+    p.v_cache_w = fuse ? static_cast<uint4*>(append->v_cache) : nullptr;
+    p.slot_mapping = fuse ? append->slot_mapping : nullptr;
     const int G = Hq / Hkv;
     if (workspace) {
         if (D == 128) return launch_g<128, true>(mk, mv, p, G, stream);

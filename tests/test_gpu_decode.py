@@ -67,6 +67,33 @@ def test_decode_step_one_call_matches_the_oracle():
         assert np.max(np.abs(got - want)) <= util.TOL[wl.dtype], wl.name
 
 
+@pytest.mark.parametrize("B,Hkv", [(40, 2), (9, 8), (600, 2)])
+def test_decode_step_leaves_the_cache_as_the_slot_mapped_write_does(B, Hkv):
+    """With few streams the step's decode kernel stores the new tokens itself (B * Hkv <= 1024), with many a separate
+    kernel does: either way the pools afterwards are bit for bit what opt_gqa_cache_append gives, skipped tokens
+    (slot -1, empty sequences) included."""
+    rng = np.random.default_rng(B)
+    lens = [int(x) for x in rng.integers(1, 700, size=B)]
+    lens[1] = 0
+    lens[2] = 1
+    lens[3] = 16
+    lens[4] = 17
+    wl = W.make_custom("fused", "bf16", Hkv * 4, Hkv, 128, 16, lens, seed=90 + B, poison=True)
+    d = util.DeviceWorkload(wl)
+    k_ref, v_ref = d.k_cache.clone(), d.v_cache.clone()
+    binding.cache_append(d.k_new, d.v_new, k_ref, v_ref, d.slot_mapping)
+    P, maxP = 256, 3
+    ws = torch.full((binding.workspace_bytes(wl.B, wl.Hq, wl.D, maxP),), 0xff, device="cuda:0", dtype=torch.uint8)
+    binding.decode_step(d.out, d.q, d.k_new, d.v_new, d.slot_mapping, d.k_cache, d.v_cache, d.block_tables,
+                        d.context_lens, d.alibi_slopes, wl.scale, partition_size=P, workspace=ws, max_partitions=maxP)
+    torch.cuda.synchronize()
+    assert binding.device_status() == 0
+    assert torch.equal(d.k_cache.view(torch.int16), k_ref.view(torch.int16))
+    assert torch.equal(d.v_cache.view(torch.int16), v_ref.view(torch.int16))
+    want = util.oracle_attention(wl)
+    assert np.max(np.abs(d.out.double().cpu().numpy() - want)) <= util.TOL["bf16"]
+
+
 def test_config4_ragged_large_batch_with_append():
     wl = W.make_config(4, poison=True)
     got, want, d = _check(wl, partition_size=512)
