@@ -49,6 +49,7 @@ constexpr int kStages = OPT_GQA_STREAM_STAGES;   // ring depth per worker
 constexpr int kCtasPerSm = OPT_GQA_STREAM_CTAS;
 constexpr int kDescSlots = 4;                    // item descriptors a worker keeps (>= items between prefetch and use)
 constexpr unsigned kFull = 0xffffffffu;
+constexpr float kMaxSlack = 8.f;                // log2 units by which a score may exceed the running reference maximum
 
 struct StreamParams {
     const __nv_bfloat16* q;
@@ -271,8 +272,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             desc[2 * (pieces & (kDescSlots - 1))] = make_int4(cur.s, cur.kvh, cur.n, first_tile_of(cur.n) + cur.jt);
             desc[2 * (pieces & (kDescSlots - 1)) + 1] = make_int4(len, obase, 0, 0);
         }
-        const int tok = (first_tile_of(cur.n) + cur.jt + lane) * kTileTok;
-        pages_nxt = lane < len ? __ldg(p.block_tables + (size_t)cur.s * p.max_blocks + tok / p.bs) : 0;
+        // the piece is streamed from its last tile backwards: page ids of its last block of 32 tiles first
+        const int blk = (len - 1) & ~31;
+        const int tok = (first_tile_of(cur.n) + cur.jt + blk + lane) * kTileTok;
+        pages_nxt = blk + lane < len ? __ldg(p.block_tables + (size_t)cur.s * p.max_blocks + tok / p.bs) : 0;
         ++pieces;
         cur.pos += len;
         cur.jt += len;
@@ -313,12 +316,13 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             for (int c = 0; c < 2; ++c)
                 sl_nxt[c] = (p.slopes && 2 * t + c < G) ? __ldg(p.slopes + d0.y * G + 2 * t + c) * kLog2e : 0.f;
             if (cur_valid()) describe_next();
-        } else if ((is_j & 31) == 0) {
-            // pieces longer than 512 tokens: the next 32 page ids
-            const int tok = (is_tile0 + is_j + lane) * kTileTok;
-            pages_cur = is_j + lane < is_ntile ? __ldg(p.block_tables + (size_t)is_s * p.max_blocks + tok / p.bs) : 0;
+        } else if (((is_ntile - 1 - is_j) & 31) == 31) {
+            // pieces longer than 512 tokens: the page ids of the block of 32 tiles below
+            const int tok = (is_tile0 + (is_ntile - 32 - is_j) + lane) * kTileTok;
+            pages_cur = __ldg(p.block_tables + (size_t)is_s * p.max_blocks + tok / p.bs);
         }
-        if (p.k_new && is_tile0 + is_j == is_last_tile) {
+        const int is_r = is_ntile - 1 - is_j;      // tile inside the piece: from the last one backwards
+        if (p.k_new && is_tile0 + is_r == is_last_tile) {
             // The step's new token of this sequence lies in the tile about to be fetched: store its K and V rows
             // of this head first (as the slot-mapped write would), and order the stores before the bulk copy.
             const long long slot = __ldg(p.slot_mapping + is_s);
@@ -336,9 +340,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
             __syncwarp();
         }
-        const int phys = __shfl_sync(kFull, pages_cur, is_j & 31);
+        const int phys = __shfl_sync(kFull, pages_cur, is_r & 31);
         if (lane == 0) {
-            const int tok = (is_tile0 + is_j) * kTileTok;
+            const int tok = (is_tile0 + is_r) * kTileTok;
             const int row = (phys * p.Hkv + is_kvh) * p.bs + tok % p.bs;       // row of the [rows, D] view
             const int st = issued % kStages;
             char* dst = ring + st * 2 * C::TILE_BYTES;
@@ -402,7 +406,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         ok = __all_sync(kFull, mbar_wait(&bars[st], (consumed / kStages) & 1, p.status));
         if (!ok) break;
 
-        const int j0 = (cs_tile0 + cs_j) * kTileTok;
+        const int j0 = (cs_tile0 + (cs_ntile - 1 - cs_j)) * kTileTok;
         const int valid = min(kTileTok, cs_n - j0);
         if (valid < kTileTok) {
             // Rows past the end of the sequence hold whatever the page held: zero the V rows so that
@@ -417,14 +421,20 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         // ---- S^T[token][head]: rows = the tile's 16 tokens, columns = heads of the group
         float sc[4] = {0.f, 0.f, 0.f, 0.f};
         {
+            // two accumulators, so that the k-steps form two dependency chains of half the length
+            float sd[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t kbase = smem_u32(kst);
             const int krow = lrow + 8 * (lmat & 1);          // matrices 0,2: tokens 0-7; 1,3: tokens 8-15
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                uint32_t a[4];
+            for (int ks = 0; ks < KS; ks += 2) {
+                uint32_t a[4], b[4];
                 ldmatrix_x4(a, kbase + swz(krow, 2 * ks + (lmat >> 1)));
+                ldmatrix_x4(b, kbase + swz(krow, 2 * ks + 2 + (lmat >> 1)));
                 mma_bf16(sc, a, qb[ks][0], qb[ks][1]);
+                mma_bf16(sd, b, qb[ks + 1][0], qb[ks + 1][1]);
             }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) sc[i] += sd[i];
         }
         // thread holds tokens j0 + g (sc[0], sc[1]) and j0 + g + 8 (sc[2], sc[3]) for heads 2t, 2t + 1
         {
@@ -438,21 +448,18 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             if (ja >= cs_n || ja < cs_start) sc[0] = sc[1] = -INFINITY;
             if (ja + 8 >= cs_n || ja + 8 < cs_start) sc[2] = sc[3] = -INFINITY;
         }
-        const float m0n = fmaxf(m0, group_max(fmaxf(sc[0], sc[2])));
-        const float m1n = fmaxf(m1, group_max(fmaxf(sc[1], sc[3])));
-        const float a0 = ex2(m0 - m0n), a1 = ex2(m1 - m1n);
-        const bool rescale = __any_sync(kFull, m0n > m0 || m1n > m1);
-        m0 = m0n;
-        m1 = m1n;
-        // p rounded to bf16 once: the same values feed the tensor core and the denominator
-        const __nv_bfloat162 pa = __floats2bfloat162_rn(ex2(sc[0] - m0n), ex2(sc[1] - m1n));   // token g
-        const __nv_bfloat162 pb = __floats2bfloat162_rn(ex2(sc[2] - m0n), ex2(sc[3] - m1n));   // token g + 8
-        const float2 fa = __bfloat1622float2(pa), fb = __bfloat1622float2(pb);
-        l0 = fmaf(l0, a0, fa.x + fb.x);
-        l1 = fmaf(l1, a1, fa.y + fb.y);
-        const uint32_t b0 = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pa));   // tokens 2t, 2t+1 of head g
-        const uint32_t b1 = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pb));   // tokens 2t+8, 2t+9
-        if (rescale) {
+        // Running maximum per head, kept lazily: the tiles of a piece come from its last one backwards, so the ALiBi
+        // term only falls after the first tile and the reference m rarely has to move.  It moves (and the
+        // accumulators are rescaled) only when some score exceeds it by more than kMaxSlack; until then p may be
+        // as large as 2^kMaxSlack, which bf16 and the fp32 sums hold as well as values below 1.
+        const float x0 = fmaxf(sc[0], sc[2]), x1 = fmaxf(sc[1], sc[3]);
+        if (__any_sync(kFull, x0 > m0 + kMaxSlack || x1 > m1 + kMaxSlack)) {
+            const float m0n = fmaxf(m0, group_max(x0)), m1n = fmaxf(m1, group_max(x1));
+            const float a0 = ex2(m0 - m0n), a1 = ex2(m1 - m1n);
+            m0 = m0n;
+            m1 = m1n;
+            l0 *= a0;
+            l1 *= a1;
 #pragma unroll
             for (int i = 0; i < MT; ++i) {
                 o[i][0] *= a0;
@@ -461,6 +468,14 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 o[i][3] *= a1;
             }
         }
+        // p rounded to bf16 once: the same values feed the tensor core and the denominator
+        const __nv_bfloat162 pa = __floats2bfloat162_rn(ex2(sc[0] - m0), ex2(sc[1] - m1));   // token g
+        const __nv_bfloat162 pb = __floats2bfloat162_rn(ex2(sc[2] - m0), ex2(sc[3] - m1));   // token g + 8
+        const float2 fa = __bfloat1622float2(pa), fb = __bfloat1622float2(pb);
+        l0 += fa.x + fb.x;
+        l1 += fa.y + fb.y;
+        const uint32_t b0 = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pa));   // tokens 2t, 2t+1 of head g
+        const uint32_t b1 = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pb));   // tokens 2t+8, 2t+9
 
         // ---- O^T[dim][head] += V^T[dim][token] * p^T[token][head]; V transposed on the fly by ldmatrix.trans
         {
@@ -502,9 +517,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             }
         }
 
-        // The slot just consumed may have been written by this warp (the zeroed rows): order those
-        // generic-proxy writes before the async-proxy copy that refills it.
-        fence_proxy_async();
+        // Where this warp wrote into the slot just consumed (the zeroed rows), order those generic-proxy writes
+        // before the async-proxy copy that refills it.  Reads need no fence: the fragments are in registers by the
+        // time the instructions that use them have been issued.
+        if (valid < kTileTok) fence_proxy_async();
         __syncwarp();
         while (issue_allowed()) issue_one();
     }
