@@ -364,6 +364,20 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         return is_piece < pieces - 1 && is_piece <= cs_piece;
     };
 
+    {
+        // While the preceding grid drains: bring what the first piece needs and that grid does not write (page ids,
+        // query rows) towards this SM, so that the first copies can be issued right after the wait.
+        const int part = cur.jt / P16;
+        int len = min((part + 1) * P16, cur.tiles) - cur.jt;
+        if (kBalanced) len = (int)min((long long)len, hi - cur.pos);
+        const int blk = (len - 1) & ~31;
+        const int tok = (first_tile_of(cur.n) + cur.jt + blk + lane) * kTileTok;
+        if (blk + lane < len)
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(p.block_tables + (size_t)cur.s * p.max_blocks + tok / p.bs));
+        if (lane < G * D * 2 / 128)
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(
+                reinterpret_cast<const char*>(p.q + ((size_t)cur.s * p.Hq + (size_t)cur.kvh * G) * D) + lane * 128));
+    }
     grid_dependency_wait();     // the cache may still be receiving this step's appended tokens
     describe_next();            // piece 0
     while (issue_allowed()) issue_one();

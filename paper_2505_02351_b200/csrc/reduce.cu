@@ -5,6 +5,8 @@
 // warp reads one partial row as one coalesced segment; the warps of the CTA take the
 // partitions round-robin (independent loads in flight instead of one dependent chain
 // over all partitions) and are folded through shared memory at the end.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace optgqa {
@@ -84,7 +86,7 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
 // rows, so that batches of many short sequences do not pay for warps with nothing to sweep).
 constexpr int kBalWarps = 8;
 
-template <typename T, int D, int WPR>
+template <typename T, int D, int WPR, int kPre>
 __global__ void __launch_bounds__(kBalWarps * 32)
 reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_out,
                        const float* __restrict__ partial_lse, const long long* __restrict__ header,
@@ -123,6 +125,21 @@ reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_ou
         po += ((size_t)r0 * G + hh) * D + lane * V;          // stride G * D
     }
 
+    // The first kPre rows of this warp's share are requested before the maximum is known: their loads travel
+    // together with those of the maximum pass instead of after it (kPre > 0 only for grids of one wave: the
+    // registers it takes would cost a many-row grid its occupancy).
+    using Vec = typename std::conditional<V == 4, float4, float2>::type;
+    float lpre[kPre > 0 ? kPre : 1];
+    Vec xpre[kPre > 0 ? kPre : 1];
+#pragma unroll
+    for (int k = 0; k < kPre; ++k) {
+        const int i = sub + k * WPR;
+        lpre[k] = -INFINITY;
+        if (i < R) {
+            lpre[k] = lse[(size_t)i * G];
+            xpre[k] = *reinterpret_cast<const Vec*>(po + (size_t)i * G * D);
+        }
+    }
     float M = -INFINITY;
     for (int i = sub * 32 + lane; i < R; i += WPR * 32) M = fmaxf(M, lse[(size_t)i * G]);
 #pragma unroll
@@ -138,26 +155,23 @@ reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_ou
 #pragma unroll
     for (int v = 0; v < V; ++v) num[v] = 0.f;
     float den = 0.f;
-#pragma unroll 4
-    for (int i = sub; i < R; i += WPR) {
-        const float l = lse[(size_t)i * G];
-        const bool piece = l > -INFINITY;                     // false for the empty numbers: their rows hold nothing
-        const float w = piece ? ex2((l - M) * kLog2e) : 0.f;
-        den += w;
-        if constexpr (V == 4) {
-            float4 x = *reinterpret_cast<const float4*>(po + (size_t)i * G * D);
-            if (!piece) x = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto add_row = [&](float l, Vec x) {
+        if (l > -INFINITY) {                                  // false for the empty numbers: their rows hold nothing
+            const float w = ex2((l - M) * kLog2e);
+            den += w;
             num[0] = fmaf(w, x.x, num[0]);
             num[1] = fmaf(w, x.y, num[1]);
-            num[2] = fmaf(w, x.z, num[2]);
-            num[3] = fmaf(w, x.w, num[3]);
-        } else {
-            float2 x = *reinterpret_cast<const float2*>(po + (size_t)i * G * D);
-            if (!piece) x = make_float2(0.f, 0.f);
-            num[0] = fmaf(w, x.x, num[0]);
-            num[1] = fmaf(w, x.y, num[1]);
+            if constexpr (V == 4) {
+                num[2] = fmaf(w, x.z, num[2]);
+                num[3] = fmaf(w, x.w, num[3]);
+            }
         }
-    }
+    };
+#pragma unroll
+    for (int k = 0; k < kPre; ++k) add_row(lpre[k], xpre[k]);
+#pragma unroll 4
+    for (int i = sub + kPre * WPR; i < R; i += WPR)
+        add_row(lse[(size_t)i * G], *reinterpret_cast<const Vec*>(po + (size_t)i * G * D));
 #pragma unroll
     for (int v = 0; v < V; ++v) s_num[warp][lane * V + v] = num[v];
     if (lane == 0) s_den[warp] = den;
@@ -202,11 +216,11 @@ int launch_reduce(void* out, const float* partial_out, const float* partial_lse,
                                       max_partitions, stream);
 }
 
-template <typename T, int D, int WPR>
+template <typename T, int D, int WPR, int kPre = 0>
 static int launch_reduce_balanced_w(void* out, const char* ws, const BalancedLayout& L, const int32_t* context_lens,
                                     int B, int Hq, int Hkv, int partition_size, int window, cudaStream_t stream) {
     const int rows = B * Hq, rpb = kBalWarps / WPR;
-    return launch_dependent(reduce_balanced_kernel<T, D, WPR>, dim3((unsigned)((rows + rpb - 1) / rpb)),
+    return launch_dependent(reduce_balanced_kernel<T, D, WPR, kPre>, dim3((unsigned)((rows + rpb - 1) / rpb)),
                             dim3(kBalWarps * 32), 0, stream, static_cast<T*>(out),
                             reinterpret_cast<const float*>(ws + L.out), reinterpret_cast<const float*>(ws + L.lse),
                             reinterpret_cast<const long long*>(ws + L.header),
@@ -219,6 +233,7 @@ static int launch_reduce_balanced_t(void* out, const char* ws, const BalancedLay
                                     int B, int Hq, int Hkv, int partition_size, int window, cudaStream_t stream) {
     // About 8192 warps in all: 8 per row for a few long rows, 1 per row for batches of many rows.
     const long long rows = (long long)B * Hq;
+    if (rows <= 256) return launch_reduce_balanced_w<T, D, 8, 12>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
     if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
     if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
     if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
