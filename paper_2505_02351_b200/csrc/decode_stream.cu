@@ -568,8 +568,11 @@ int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams&
     }
     const int sms = sm_count();
     if (sms <= 0) return OPT_GQA_ERR_CUDA;
-    // One resident wave; never more workers than there could be partitions, nor than the workspace has room for.
-    const long long items = (long long)p.B * p.Hkv * p.max_partitions;
+    // One resident wave; never more workers than there could be units of work (whole partitions, or 16-token tiles
+    // in the balanced split, whose ranges are cut at tile granularity), nor than the workspace has room for.  In
+    // the balanced split a grid that leaves some SMs with one CTA and others with two would undo the balance.
+    long long items = (long long)p.B * p.Hkv * p.max_partitions;
+    if (kBalanced) items *= p.partition_size / kTileTok;
     long long ctas = (items + kWarps - 1) / kWarps;
     if (ctas > (long long)sms * kCtasPerSm) ctas = (long long)sms * kCtasPerSm;
     if (ctas > kBalancedMaxWorkers / kWarps) ctas = kBalancedMaxWorkers / kWarps;
