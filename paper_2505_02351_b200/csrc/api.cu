@@ -317,19 +317,43 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
 }
 
 namespace {
-// Six host arrays copied to device staging by ONE kernel that reads pinned host memory directly (32-bit words).
+// Six host arrays copied to device staging by ONE kernel that reads pinned host memory directly, in words of
+// type V (16 bytes where every array allows it, else 4).  The arrays are numbered through as one range of words;
+// a thread requests up to four words before it stores any, so the whole step's input crosses the bus in about one
+// round trip instead of one per array.
 struct HostGather {
-    const uint32_t* src[6];
-    uint32_t* dst[6];
-    unsigned words[6];
+    const void* src[6];
+    void* dst[6];
+    unsigned first[7];      // first[a] .. first[a + 1]: the words of array a in the joint numbering
 };
 
+extern "C++" {
+template <typename V>
 __global__ void __launch_bounds__(256) gather_host_kernel(const HostGather g) {
-    const unsigned tid = blockIdx.x * blockDim.x + threadIdx.x, nthreads = gridDim.x * blockDim.x;
+    const unsigned tid = blockIdx.x * blockDim.x + threadIdx.x, nthreads = gridDim.x * blockDim.x, total = g.first[6];
+    for (unsigned base = tid; base < total; base += 4 * nthreads) {
+        V v[4];
+        int arr[4];
 #pragma unroll
-    for (int a = 0; a < 6; ++a)
-        for (unsigned i = tid; i < g.words[a]; i += nthreads) g.dst[a][i] = g.src[a][i];
+        for (int u = 0; u < 4; ++u) {
+            const unsigned i = base + u * nthreads;
+            arr[u] = -1;
+            if (i < total) {
+                int a = 0;
+#pragma unroll
+                for (int k = 1; k < 6; ++k) a += i >= g.first[k];
+                arr[u] = a;
+                v[u] = static_cast<const V*>(g.src[a])[i - g.first[a]];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned i = base + u * nthreads;
+            if (arr[u] >= 0) static_cast<V*>(g.dst[arr[u]])[i - g.first[arr[u]]] = v[u];
+        }
+    }
 }
+}  // extern "C++"
 
 // The device-side address of pinned (page-locked, mapped) host memory, or nullptr for pageable memory.
 const void* device_view(const void* host) {
@@ -394,18 +418,28 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
     const size_t off[6] = {L.q, L.k_new, L.v_new, L.slots, L.tables, L.lens};
     const size_t bytes[6] = {qb, kb, kb, (size_t)B * 8, (size_t)B * max_blocks_per_seq * 4, (size_t)B * 4};
     HostGather g;
-    bool pinned = true;
+    bool pinned = true, wide = true;
     for (int a = 0; a < 6; ++a) {
         const void* dv = device_view(src[a]);
-        pinned &= dv != nullptr && bytes[a] % 4 == 0 && bytes[a] / 4 <= 0xffffffffull;
-        g.src[a] = static_cast<const uint32_t*>(dv);
-        g.dst[a] = reinterpret_cast<uint32_t*>(st + off[a]);
-        g.words[a] = (unsigned)(bytes[a] / 4);
+        pinned &= dv != nullptr && bytes[a] % 4 == 0;
+        wide &= bytes[a] % 16 == 0 && (reinterpret_cast<uintptr_t>(dv) & 15u) == 0;
+        g.src[a] = dv;
+        g.dst[a] = st + off[a];
     }
+    const size_t word = wide ? 16 : 4;
+    size_t words = 0;
+    for (int a = 0; a < 6; ++a) {
+        g.first[a] = (unsigned)words;
+        words += bytes[a] / word;
+    }
+    pinned &= words <= 0x7fffffffull;
+    g.first[6] = (unsigned)words;
     void* out_dev = pinned ? const_cast<void*>(device_view(out_host)) : nullptr;
     pinned &= out_dev != nullptr && (reinterpret_cast<uintptr_t>(out_dev) & 15u) == 0;
     if (pinned) {
-        gather_host_kernel<<<32, 256, 0, cs>>>(g);
+        const unsigned ctas = (unsigned)((words + 255) / 256 < 148 ? (words + 255) / 256 : 148);
+        if (wide) gather_host_kernel<uint4><<<ctas, 256, 0, cs>>>(g);
+        else gather_host_kernel<uint32_t><<<ctas, 256, 0, cs>>>(g);
         if (cudaGetLastError() != cudaSuccess) return OPT_GQA_ERR_CUDA;
     } else {
         bool ok = true;
