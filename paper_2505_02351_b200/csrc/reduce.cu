@@ -234,10 +234,11 @@ static int launch_reduce_balanced_t(void* out, const char* ws, const BalancedLay
     // About 8192 warps in all: 8 per row for a few long rows, 1 per row for batches of many rows.
     const long long rows = (long long)B * Hq;
     if (rows <= 256) return launch_reduce_balanced_w<T, D, 8, 12>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    return launch_reduce_balanced_w<T, D, 1>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    // Batches of many rows are mostly short rows (a few pieces each): four preloaded rows cover them in one round trip.
+    return launch_reduce_balanced_w<T, D, 1, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
 }
 
 int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
