@@ -92,6 +92,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
 
     grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
+    const uint64_t read_once = l2_policy_evict_first();     // every K/V byte is read exactly once
     const int part = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;      // fragment row (query head of the group) and column pair
@@ -147,8 +148,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             mbar_expect_tx(bar, 2 * C::TILE_BYTES);
 #pragma unroll
             for (int b = 0; b < C::NBOX; ++b) {
-                tma_load_2d(dst + b * C::BOX_BYTES, &map_k, b * 64, row, bar);
-                tma_load_2d(dst + C::TILE_BYTES + b * C::BOX_BYTES, &map_v, b * 64, row, bar);
+                tma_load_2d_hint(dst + b * C::BOX_BYTES, &map_k, b * 64, row, bar, read_once);
+                tma_load_2d_hint(dst + C::TILE_BYTES + b * C::BOX_BYTES, &map_v, b * 64, row, bar, read_once);
             }
         }
     };
