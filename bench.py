@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 DEFAULT_PARTITION = {2: 256, 3: 512, 4: 512}
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised
 # under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {3: 378_693_888 + 6_016_256}   # profiles/decode_stream_cfg3.md
+NCU_TRAFFIC_BYTES = {3: 378_693_376 + 3_752_704}   # profiles/decode_stream_cfg3.md
 
 
 # ----------------------------------------------------------------------------- distributed plumbing

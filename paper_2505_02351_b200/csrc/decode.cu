@@ -138,6 +138,7 @@ decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(128) char smem[];
 
     grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
+    const uint64_t read_once = l2_policy_evict_first();     // every K/V byte is read exactly once
     const int part = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, c = lane & 15;
@@ -196,8 +197,8 @@ decode_kernel(const DecodeParams p) {
             char* dst = ring + (k % kStages) * 2 * C::TILE_BYTES;
             uint64_t* bar = &bars[k % kStages];
             mbar_expect_tx(bar, 2 * C::TILE_BYTES);
-            bulk_g2s(dst, p.k_cache + off, C::TILE_BYTES, bar);
-            bulk_g2s(dst + C::TILE_BYTES, p.v_cache + off, C::TILE_BYTES, bar);
+            bulk_g2s_hint(dst, p.k_cache + off, C::TILE_BYTES, bar, read_once);
+            bulk_g2s_hint(dst + C::TILE_BYTES, p.v_cache + off, C::TILE_BYTES, bar, read_once);
         }
     };
 

@@ -137,6 +137,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 
     grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
     const uint64_t read_once = l2_policy_evict_first();     // every K/V byte is read exactly once
+    const uint64_t keep = l2_policy_evict_last();           // the pieces are read by the merge that follows
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const int P = p.partition_size, P16 = P / kTileTok;    // tiles per full partition
@@ -515,20 +516,20 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 float* po = p.partial_out + row * D;
 #pragma unroll
                 for (int i = 0; i < MT; ++i) {
-                    po[16 * i + g] = o[i][0] * i0;
-                    po[16 * i + 8 + g] = o[i][2] * i0;
+                    st_global_hint(po + 16 * i + g, o[i][0] * i0, keep);
+                    st_global_hint(po + 16 * i + 8 + g, o[i][2] * i0, keep);
                 }
-                if (g == 0) p.partial_lse[row] = (m0 + lg2(L0)) * kLn2;
+                if (g == 0) st_global_hint(p.partial_lse + row, (m0 + lg2(L0)) * kLn2, keep);
             }
             if (2 * t + 1 < G) {
                 const size_t row = (size_t)cs_obase + (size_t)(2 * t + 1) * ostride;
                 float* po = p.partial_out + row * D;
 #pragma unroll
                 for (int i = 0; i < MT; ++i) {
-                    po[16 * i + g] = o[i][1] * i1;
-                    po[16 * i + 8 + g] = o[i][3] * i1;
+                    st_global_hint(po + 16 * i + g, o[i][1] * i1, keep);
+                    st_global_hint(po + 16 * i + 8 + g, o[i][3] * i1, keep);
                 }
-                if (g == 0) p.partial_lse[row] = (m1 + lg2(L1)) * kLn2;
+                if (g == 0) st_global_hint(p.partial_lse + row, (m1 + lg2(L1)) * kLn2, keep);
             }
         }
 

@@ -18,12 +18,16 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
         : "memory");
 }
 
-// L2 policy for data that is read once: its lines are the first to be evicted, so a stream of K/V tiles does not
-// push out what will be read again (the partitions' partial results waiting for their merge).
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+// L2 policy for data that is written now and read again soon (by the next kernel of the stream): its lines are the
+// last to be evicted.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
     uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
     return pol;
+}
+
+__device__ __forceinline__ void st_global_hint(float* p, float v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(policy) : "memory");
 }
 
 // tma_load_2d with an L2 cache policy (see l2_policy_evict_first).
