@@ -273,3 +273,19 @@ def test_decode_step_from_host_buffers(pinned):
         assert binding.device_status() == 0
         want = util.oracle_attention(wl)
         assert np.max(np.abs(hout.double().numpy() - want)) <= util.TOL[wl.dtype], (wl.name, pinned)
+
+
+@pytest.mark.parametrize("scale", [0.0, 0.02, 1.0, 6.0])
+@pytest.mark.parametrize("slope", ["usual", "zero", "steep", "negative"])
+def test_reference_maximum_that_moves_inside_a_piece(scale, slope):
+    """The streaming kernel walks a piece from its last tile backwards and moves its reference maximum only when a
+    score exceeds it by 2^8.  Large scales make the maximum jump at arbitrary tiles, steep or negative slopes make it
+    move at every tile or never: the result must be the oracle's in every case."""
+    Hq = 8
+    slopes = {"usual": None, "zero": torch.zeros(Hq), "steep": torch.full((Hq,), 3.0),
+              "negative": -torch.logspace(-3, -1, Hq)}[slope]
+    wl = W.make_custom("maxmove", "bf16", Hq, 2, 128, 16, [2100, 515, 16, 1, 700], seed=29, poison=True,
+                       slopes=slopes, scale=scale)
+    for P in (512, 64):
+        _check(wl, partition_size=P, balanced=True)
+    _check(wl, partition_size=128)
