@@ -289,3 +289,31 @@ def test_reference_maximum_that_moves_inside_a_piece(scale, slope):
     for P in (512, 64):
         _check(wl, partition_size=P, balanced=True)
     _check(wl, partition_size=128)
+
+
+def test_host_step_called_repeatedly_reads_the_buffers_anew():
+    """Repeated calls of opt_gqa_decode_step_host with the same buffers, on a stream of the caller's: every call
+    reads what the pinned buffers hold at that moment and leaves its result in out_host."""
+    wl = W.make_custom("hoststeps", "bf16", 32, 4, 128, 16, [1500, 700, 40, 1], seed=31)
+    d = util.DeviceWorkload(wl)
+    pin = lambda t: t.contiguous().pin_memory()
+    hq, hk, hv = pin(wl.q), pin(wl.k_new), pin(wl.v_new)
+    hs, ht, hl = pin(wl.slot_mapping), pin(wl.block_tables), pin(wl.context_lens)
+    hout = pin(torch.full_like(wl.q, float("nan")))
+    P, maxP = 512, 3
+    staging = torch.empty(binding.step_staging_bytes(wl.B, wl.Hq, wl.Hkv, wl.D, wl.max_blocks, torch.bfloat16),
+                          dtype=torch.uint8, device="cuda:0")
+    ws = torch.empty(binding.workspace_bytes(wl.B, wl.Hq, wl.D, maxP), dtype=torch.uint8, device="cuda:0")
+    stream = torch.cuda.Stream()
+    gen = torch.Generator().manual_seed(5)
+    for call in range(5):
+        q = torch.randn(wl.q.shape, generator=gen).to(torch.bfloat16)
+        hq.copy_(q)
+        hout.fill_(float("nan"))
+        with torch.cuda.stream(stream):
+            binding.decode_step_host(hout, hq, hk, hv, hs, ht, hl, staging, d.k_cache, d.v_cache, d.alibi_slopes,
+                                     wl.scale, partition_size=P, workspace=ws, max_partitions=maxP)
+        stream.synchronize()
+        assert binding.device_status() == 0
+        want = util.oracle_attention(W.Workload(**{**wl.__dict__, "q": q}))
+        assert np.max(np.abs(hout.double().numpy() - want)) <= util.TOL["bf16"], call
