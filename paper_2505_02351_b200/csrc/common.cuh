@@ -223,6 +223,10 @@ int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache
                          float* partial_out, float* partial_lse, void* workspace, int max_partitions, int window,
                          int* device_status, cudaStream_t stream, const FusedAppend* append = nullptr);
 
+// Workers (warps) of the grid that launch_decode_stream uses for the balanced split of these sizes on the current
+// device; 0 if the device cannot be queried.
+long long stream_grid_workers(int B, int Hkv, int max_partitions, int partition_size);
+
 // Merge of the balanced split's pieces (reduce.cu).
 int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
                            int D, int partition_size, int max_partitions, int window, int dtype, cudaStream_t stream);

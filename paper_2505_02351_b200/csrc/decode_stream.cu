@@ -556,6 +556,20 @@ int sm_count() {
     return counts[dev];
 }
 
+// One resident wave; never more workers than there could be units of work (whole partitions, or 16-token tiles in the
+// balanced split, whose ranges are cut at tile granularity), nor than the workspace has room for.  In the balanced
+// split a grid that leaves some SMs with one CTA and others with two would undo the balance.
+long long stream_grid_ctas(int B, int Hkv, int max_partitions, int partition_size, bool balanced) {
+    const int sms = sm_count();
+    if (sms <= 0) return 0;
+    long long items = (long long)B * Hkv * max_partitions;
+    if (balanced) items *= partition_size / kTileTok;
+    long long ctas = (items + kWarps - 1) / kWarps;
+    if (ctas > (long long)sms * kCtasPerSm) ctas = (long long)sms * kCtasPerSm;
+    if (ctas > kBalancedMaxWorkers / kWarps) ctas = kBalancedMaxWorkers / kWarps;
+    return ctas;
+}
+
 template <int D, int G, bool kBalanced>
 int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams& p, cudaStream_t stream) {
     using C = StreamCfg<D>;
@@ -568,16 +582,8 @@ int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams&
             return OPT_GQA_ERR_CUDA;
         configured[dev] = true;
     }
-    const int sms = sm_count();
-    if (sms <= 0) return OPT_GQA_ERR_CUDA;
-    // One resident wave; never more workers than there could be units of work (whole partitions, or 16-token tiles
-    // in the balanced split, whose ranges are cut at tile granularity), nor than the workspace has room for.  In
-    // the balanced split a grid that leaves some SMs with one CTA and others with two would undo the balance.
-    long long items = (long long)p.B * p.Hkv * p.max_partitions;
-    if (kBalanced) items *= p.partition_size / kTileTok;
-    long long ctas = (items + kWarps - 1) / kWarps;
-    if (ctas > (long long)sms * kCtasPerSm) ctas = (long long)sms * kCtasPerSm;
-    if (ctas > kBalancedMaxWorkers / kWarps) ctas = kBalancedMaxWorkers / kWarps;
+    const long long ctas = stream_grid_ctas(p.B, p.Hkv, p.max_partitions, p.partition_size, kBalanced);
+    if (ctas <= 0) return OPT_GQA_ERR_CUDA;
     return launch_dependent(decode_stream_kernel<D, G, kBalanced>, dim3((unsigned)ctas), dim3(kWarps * 32), C::SMEM,
                             stream, mk, mv, p);
 }
@@ -594,6 +600,10 @@ int launch_g(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams& p
 }
 
 }  // namespace
+
+long long stream_grid_workers(int B, int Hkv, int max_partitions, int partition_size) {
+    return stream_grid_ctas(B, Hkv, max_partitions, partition_size, true) * kWarps;
+}
 
 // workspace == nullptr: one partial result per partition in partial_out / partial_lse ([B, Hq, max_partitions, ...]).
 // Otherwise the balanced split: pieces and bookkeeping go to `workspace` (see balanced_layout).

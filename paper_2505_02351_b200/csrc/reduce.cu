@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(kBalWarps * 32)
 reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_out,
                        const float* __restrict__ partial_lse, const long long* __restrict__ header,
                        const long long* __restrict__ seq_info, const int32_t* __restrict__ context_lens, int rows,
-                       int Hq, int Hkv, int partition_size, int window) {
+                       int Hq, int Hkv, int partition_size, int window, int B, long long grid_workers) {
     constexpr int V = D / 32;             // columns per lane
     constexpr int RPB = kBalWarps / WPR;  // rows per CTA
     __shared__ float s_num[kBalWarps][D];
@@ -108,15 +108,42 @@ reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_ou
     const int P16 = partition_size / 16;
     const int tiles = (n + 15) / 16 - (window > 0 ? max(0, n - window) / 16 : 0);
     const int np = (tiles + P16 - 1) / P16;
+    // With at most 32 sequences a warp works out the decode grid's bookkeeping (tiles and partitions before the
+    // sequence, tiles in all, ranges) from the lengths itself, while the decode grid is still running, instead of
+    // reading it from the workspace afterwards: one dependent round trip less between the two grids.
+    const bool own_counts = grid_workers > 0 && B <= 32;
+    long long total = 0, workers = 1, tiles_before = 0, parts_before = 0;
+    if (own_counts) {
+        const int nl = lane < B ? context_lens[lane] : 0;
+        const int tl = (nl + 15) / 16 - (window > 0 ? max(0, nl - window) / 16 : 0);
+        int it = tl, ip = (tl + P16 - 1) / P16;
+#pragma unroll
+        for (int o2 = 1; o2 < 32; o2 <<= 1) {
+            const int vt = __shfl_up_sync(0xffffffffu, it, o2), vp = __shfl_up_sync(0xffffffffu, ip, o2);
+            if (lane >= o2) {
+                it += vt;
+                ip += vp;
+            }
+        }
+        total = (long long)__shfl_sync(0xffffffffu, it, 31) * Hkv;
+        tiles_before = __shfl_sync(0xffffffffu, it, s) - tiles;
+        parts_before = __shfl_sync(0xffffffffu, ip, s) - np;
+        workers = total < grid_workers ? (total > 0 ? total : 1) : grid_workers;
+    }
     grid_dependency_wait();                                 // the pieces come from the decode grid
 
     int R = 0;
     const float* lse = partial_lse;
     const float* po = partial_out;
     if (np > 0) {
-        const long long total = header[0], workers = header[1];
-        const long long first_tile = seq_info[2 * s] * Hkv + (long long)kvh * tiles;
-        const long long first_part = seq_info[2 * s + 1] * Hkv + (long long)kvh * np;
+        if (!own_counts) {
+            total = header[0];
+            workers = header[1];
+            tiles_before = seq_info[2 * s];
+            parts_before = seq_info[2 * s + 1];
+        }
+        const long long first_tile = tiles_before * Hkv + (long long)kvh * tiles;
+        const long long first_part = parts_before * Hkv + (long long)kvh * np;
         // worker whose range [floor(T w / W), floor(T (w + 1) / W)) holds tile x: floor(((x + 1) W - 1) / T)
         const long long r0 = first_part + ((first_tile + 1) * workers - 1) / total;
         const long long r1 = first_part + np - 1 + ((first_tile + tiles) * workers - 1) / total;
@@ -218,40 +245,44 @@ int launch_reduce(void* out, const float* partial_out, const float* partial_lse,
 
 template <typename T, int D, int WPR, int kPre = 0>
 static int launch_reduce_balanced_w(void* out, const char* ws, const BalancedLayout& L, const int32_t* context_lens,
-                                    int B, int Hq, int Hkv, int partition_size, int window, cudaStream_t stream) {
+                                    int B, int Hq, int Hkv, int partition_size, int window, long long gw,
+                                    cudaStream_t stream) {
     const int rows = B * Hq, rpb = kBalWarps / WPR;
     return launch_dependent(reduce_balanced_kernel<T, D, WPR, kPre>, dim3((unsigned)((rows + rpb - 1) / rpb)),
                             dim3(kBalWarps * 32), 0, stream, static_cast<T*>(out),
                             reinterpret_cast<const float*>(ws + L.out), reinterpret_cast<const float*>(ws + L.lse),
                             reinterpret_cast<const long long*>(ws + L.header),
                             reinterpret_cast<const long long*>(ws + L.seq_info), context_lens, rows, Hq, Hkv,
-                            partition_size, window);
+                            partition_size, window, B, gw);
 }
 
 template <typename T, int D>
 static int launch_reduce_balanced_t(void* out, const char* ws, const BalancedLayout& L, const int32_t* context_lens,
-                                    int B, int Hq, int Hkv, int partition_size, int window, cudaStream_t stream) {
+                                    int B, int Hq, int Hkv, int partition_size, int window, long long gw,
+                                    cudaStream_t stream) {
     // About 8192 warps in all: 8 per row for a few long rows, 1 per row for batches of many rows.
     const long long rows = (long long)B * Hq;
-    if (rows <= 256) return launch_reduce_balanced_w<T, D, 8, 12>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    if (rows <= 256) return launch_reduce_balanced_w<T, D, 8, 12>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
+    if (rows <= 1024) return launch_reduce_balanced_w<T, D, 8, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
+    if (rows <= 2048) return launch_reduce_balanced_w<T, D, 4, 2>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
+    if (rows <= 4096) return launch_reduce_balanced_w<T, D, 2, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
     // Batches of many rows are mostly short rows (a few pieces each): four preloaded rows cover them in one round trip.
-    return launch_reduce_balanced_w<T, D, 1, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    return launch_reduce_balanced_w<T, D, 1, 4>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
 }
 
 int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
                            int D, int partition_size, int max_partitions, int window, int dtype, cudaStream_t stream) {
     const BalancedLayout L = balanced_layout(B, Hq, Hkv, D, max_partitions);
     const char* ws = static_cast<const char*>(workspace);
+    // workers of the decode grid that filled the workspace (0: unknown, the kernel reads the count from the workspace)
+    const long long gw = stream_grid_workers(B, Hkv, max_partitions, partition_size);
     if (dtype == OPT_GQA_BF16) {
         if (D == 128)
-            return launch_reduce_balanced_t<__nv_bfloat16, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-        return launch_reduce_balanced_t<__nv_bfloat16, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+            return launch_reduce_balanced_t<__nv_bfloat16, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
+        return launch_reduce_balanced_t<__nv_bfloat16, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
     }
-    if (D == 128) return launch_reduce_balanced_t<float, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
-    return launch_reduce_balanced_t<float, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, stream);
+    if (D == 128) return launch_reduce_balanced_t<float, 128>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
+    return launch_reduce_balanced_t<float, 64>(out, ws, L, context_lens, B, Hq, Hkv, partition_size, window, gw, stream);
 }
 
 }  // namespace optgqa
