@@ -74,10 +74,8 @@ static int decode_checked(bool allow_tensor_cores, void* out, const void* q, con
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    if (allow_tensor_cores && dtype == OPT_GQA_BF16 && partition_size > 0)
-        return launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
-                                    scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out, partial_lse,
-                                    nullptr, max_partitions, 0, status, cs);
+    // bf16: one CTA per (sequence, KV head, partition) -- whole partitions as work items are balanced best by the
+    // hardware's own CTA scheduler (the persistent streaming kernel needs pieces smaller than a partition to balance)
     if (allow_tensor_cores && dtype == OPT_GQA_BF16)
         return launch_decode_tc(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                                 alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,

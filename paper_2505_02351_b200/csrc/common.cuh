@@ -214,8 +214,8 @@ struct FusedAppend {
     const int64_t* slot_mapping;    // [B]; negative: nothing to store
 };
 
-// bf16, partition_size > 0: persistent streaming kernel, one worker per warp (decode_stream.cu).
-// workspace == nullptr writes one partial per partition to partial_out / partial_lse; otherwise the balanced split.
+// bf16, partition_size > 0, balanced split into `workspace`: persistent streaming kernel, one worker per warp
+// (decode_stream.cu).  partial_out / partial_lse are unused (one partial per partition is launch_decode_tc's job).
 // append != nullptr (balanced split only): see FusedAppend.
 int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,

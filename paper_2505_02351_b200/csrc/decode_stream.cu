@@ -605,8 +605,9 @@ long long stream_grid_workers(int B, int Hkv, int max_partitions, int partition_
     return stream_grid_ctas(B, Hkv, max_partitions, partition_size, true) * kWarps;
 }
 
-// workspace == nullptr: one partial result per partition in partial_out / partial_lse ([B, Hq, max_partitions, ...]).
-// Otherwise the balanced split: pieces and bookkeeping go to `workspace` (see balanced_layout).
+// The balanced split: pieces and bookkeeping go to `workspace` (see balanced_layout).  (The kernel can also own whole
+// partitions and write one partial result per partition to partial_out / partial_lse -- kBalanced = false -- but
+// whole partitions are balanced better by one CTA per partition, decode_tc.cu, which is what the library launches.)
 int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                          int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
@@ -652,13 +653,9 @@ int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache
     p.v_cache_w = fuse ? static_cast<uint4*>(append->v_cache) : nullptr;
     p.slot_mapping = fuse ? append->slot_mapping : nullptr;
     const int G = Hq / Hkv;
-    if (workspace) {
-        if (D == 128) return launch_g<128, true>(mk, mv, p, G, stream);
-        if (D == 64) return launch_g<64, true>(mk, mv, p, G, stream);
-    } else {
-        if (D == 128) return launch_g<128, false>(mk, mv, p, G, stream);
-        if (D == 64) return launch_g<64, false>(mk, mv, p, G, stream);
-    }
+    if (!workspace) return OPT_GQA_ERR_NULL;    // one partial per partition: decode_tc.cu (one CTA per partition)
+    if (D == 128) return launch_g<128, true>(mk, mv, p, G, stream);
+    if (D == 64) return launch_g<64, true>(mk, mv, p, G, stream);
     return OPT_GQA_ERR_SHAPE;
 }
 

@@ -93,6 +93,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
 
     grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
     const uint64_t read_once = l2_policy_evict_first();     // every K/V byte is read exactly once
+    const uint64_t keep = l2_policy_evict_last();           // the partial results are read by the merge that follows
     const int part = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;      // fragment row (query head of the group) and column pair
@@ -302,8 +303,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         const float r = num / den;
         const size_t row = (size_t)s * p.Hq + (size_t)kvh * G + hg;
         if (split) {
-            p.partial_out[(row * p.max_partitions + part) * D + d] = r;
-            if (d == 0) p.partial_lse[row * p.max_partitions + part] = (M + log2f(den)) * kLn2;
+            st_global_hint(p.partial_out + (row * p.max_partitions + part) * D + d, r, keep);
+            if (d == 0) st_global_hint(p.partial_lse + row * p.max_partitions + part, (M + log2f(den)) * kLn2, keep);
         } else {
             static_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(r);
         }

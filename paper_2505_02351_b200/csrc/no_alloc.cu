@@ -73,9 +73,9 @@ extern "C" int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q,
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     int rc;
     if (dtype == OPT_GQA_BF16)
-        rc = launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
-                                  scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out, partial_lse,
-                                  nullptr, max_partitions, 0, status, cs);
+        rc = launch_decode_tc(nullptr, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+                              alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
+                              partial_lse, max_partitions, status, cs);
     else
         rc = launch_decode(nullptr, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                            alibi_slopes, scale, B, Hq, Hkv, D, bs, partition_size, partial_out, partial_lse,
