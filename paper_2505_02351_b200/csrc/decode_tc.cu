@@ -21,19 +21,18 @@ namespace optgqa {
 
 namespace {
 
-#ifndef OPT_GQA_TC_WARPS
-#define OPT_GQA_TC_WARPS 4
-#endif
 #ifndef OPT_GQA_TC_STAGES
 #define OPT_GQA_TC_STAGES 2
 #endif
-#ifndef OPT_GQA_TC_CTAS
-#define OPT_GQA_TC_CTAS 3
-#endif
+// Warps per CTA (each with a private ring) and CTAs per SM the register budget is held to, for the two uses of the
+// kernel.  One CTA per (sequence, KV head) has the whole context to itself: eight warps, one CTA per SM.  One CTA per
+// (sequence, KV head, partition) has a few hundred tokens: two warps, six CTAs per SM, so that the CTA scheduler has
+// many small items to even out.  (Measured: single pass on 256 streams of 512-2048 tokens 35.3 us with 4 warps x 3
+// CTAs, 30.6 with 8 x 1; one partial per 512-token partition on long contexts 75.0 with 4 x 3, 71.8 with 2 x 6.)
+constexpr int kWarpsSingle = 8, kCtasSingle = 1;
+constexpr int kWarpsSplit = 2, kCtasSplit = 6;
 constexpr int kTileTok = 16;                 // tokens per tile (one ring stage holds a K tile and a V tile)
-constexpr int kWarps = OPT_GQA_TC_WARPS;     // warps per CTA, each with a private ring
 constexpr int kStages = OPT_GQA_TC_STAGES;   // ring depth per warp
-constexpr int kMinCtas = OPT_GQA_TC_CTAS;    // CTAs per SM the register budget is held to
 constexpr unsigned kFull = 0xffffffffu;
 
 struct TcParams {
@@ -54,7 +53,7 @@ struct TcParams {
     int max_partitions;
 };
 
-template <int D, int G>
+template <int D, int G, int kWarps>
 struct TcCfg {
     static constexpr int NBOX = D / 64;                   // 128-byte-wide boxes per token row
     static constexpr int BOX_BYTES = kTileTok * 128;      // 16 rows x 128 B
@@ -81,11 +80,11 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
     return (uint32_t)((chunk >> 3) * (kTileTok * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
-template <int D, int G>
+template <int D, int G, int kWarps, int kMinCtas>
 __global__ void __launch_bounds__(kWarps * 32, kMinCtas)
 decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                  const TcParams p) {
-    using C = TcCfg<D, G>;
+    using C = TcCfg<D, G, kWarps>;
     constexpr int KS = D / 16;    // k-steps of q k^T
     constexpr int NT = D / 8;     // n-tiles of p V
     extern __shared__ char smem_raw[];
@@ -311,19 +310,27 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     }
 }
 
-template <int D, int G>
-int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, int B, cudaStream_t stream) {
-    using C = TcCfg<D, G>;
+template <int D, int G, int kWarps, int kMinCtas>
+int launch_shape(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, int B, cudaStream_t stream) {
+    using C = TcCfg<D, G, kWarps>;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
     if (dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(decode_tc_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_tc_kernel<D, G, kWarps, kMinCtas>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 C::SMEM) != cudaSuccess)
             return OPT_GQA_ERR_CUDA;
         configured[dev] = true;
     }
     dim3 grid(p.partition_size > 0 ? p.max_partitions : 1, p.Hkv, B);
-    return launch_dependent(decode_tc_kernel<D, G>, grid, dim3(kWarps * 32), C::SMEM, stream, mk, mv, p);
+    return launch_dependent(decode_tc_kernel<D, G, kWarps, kMinCtas>, grid, dim3(kWarps * 32), C::SMEM, stream, mk, mv,
+                            p);
+}
+
+template <int D, int G>
+int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, int B, cudaStream_t stream) {
+    if (p.partition_size > 0) return launch_shape<D, G, kWarpsSplit, kCtasSplit>(mk, mv, p, B, stream);
+    return launch_shape<D, G, kWarpsSingle, kCtasSingle>(mk, mv, p, B, stream);
 }
 
 template <int D>
