@@ -195,6 +195,15 @@ class DeviceBatch:
                 self.partial_out.data_ptr() if self.P else None, self.partial_lse.data_ptr() if self.P else None,
                 self.maxP, self.dt, stream)
 
+    def args_decode_plain(self, i, stream):
+        """opt_gqa_paged_attention_decode: single pass (P = 0) or one partial per partition."""
+        wl = self.wl
+        return (self.out.data_ptr(), self.q.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(),
+                self.tables.data_ptr(), wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B,
+                wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, self.P,
+                self.partial_out.data_ptr() if self.P else None, self.partial_lse.data_ptr() if self.P else None,
+                self.maxP, self.dt, stream)
+
     def args_reduce(self, stream):
         wl = self.wl
         if self.balanced:
@@ -368,6 +377,49 @@ def projection_report(dev, only=None) -> dict:
                      "timing": f"median over 20 replays of a graph of {per_graph} launches, CUDA events around each replay",
                      "peak_kind": f"of {kind}"}
         del packed, graph
+        torch.cuda.empty_cache()
+    return out
+
+
+def entry_point_report(dev, peak) -> dict:
+    """Side measurement of the decode entry points that a step does not use: opt_gqa_paged_attention_decode with one
+    partial per partition followed by opt_gqa_paged_attention_reduce, and the single pass (partition_size 0).
+    Back-to-back calls over rotating pool copies, CUDA events around the whole run."""
+    import torch
+
+    from paper_2505_02351_b200 import workloads as W
+
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+    out = {}
+    for cfg, P in ((3, 512), (2, 0), (4, 0)):
+        wl = W.make_config(cfg)
+        b = DeviceBatch(wl, P, 2, dev)
+        lib = b.lib
+        a_dec = [b.args_decode_plain(i, sh) for i in range(2)]
+        a_red = (b.out.data_ptr(), b.partial_out.data_ptr(), b.partial_lse.data_ptr(), b.lens.data_ptr(), wl.B, wl.Hq,
+                 wl.D, P, b.maxP, b.dt, sh) if P else None
+
+        def call(i):
+            check(lib.opt_gqa_paged_attention_decode(*a_dec[i % 2]), "decode")
+            if P:
+                check(lib.opt_gqa_paged_attention_reduce(*a_red), "reduce")
+
+        for i in range(10):
+            call(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 100
+        e0.record(stream)
+        for i in range(n):
+            call(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / n
+        gbs = b.algorithmic_bytes() / us / 1e3
+        key = f"{wl.name}: " + ("decode with one partial per partition + reduce" if P else "single-pass decode")
+        out[key] = {"us_per_call": us, "GBs": gbs, "frac_of_peak": gbs / peak, "partition_size": P}
+        del b, wl
         torch.cuda.empty_cache()
     return out
 
@@ -728,6 +780,7 @@ def main():
                               "frac_of_peak": a2 / (d_ms * 1e-3) / 1e9 / peak, "partition_size": b2.P}
             del b2, w2
             torch.cuda.empty_cache()
+        extra["other_decode_entry_points"] = entry_point_report(dev, peak)
         extra[W.CONFIG_NAMES[5]] = prefill_report(dev, 20, 3)
         extra["int4_qkv_projection"] = projection_report(dev)
         line["other_workloads"] = extra
