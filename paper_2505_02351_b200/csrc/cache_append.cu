@@ -18,6 +18,7 @@ cache_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v
     long long th = i / row_vecs;  // token * Hkv + head
     int h = (int)(th % Hkv);
     long long t = th / Hkv;
+    grid_dependency_wait();     // the new rows and the slots may come from the preceding grid, which may also still read the cache
     long long slot = slot_mapping[t];
     if (slot < 0) return;
     long long page = slot / bs;
@@ -35,10 +36,11 @@ int launch_cache_append(const void* k_new, const void* v_new, void* k_cache, voi
     const long long total = (long long)T * Hkv * row_vecs;
     const int threads = 256;
     const long long blocks = (total + threads - 1) / threads;
-    cache_append_kernel<<<(unsigned)blocks, threads, 0, stream>>>(
-        static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), static_cast<uint4*>(k_cache),
-        static_cast<uint4*>(v_cache), slot_mapping, total, Hkv, row_vecs, bs);
-    return cudaGetLastError() == cudaSuccess ? OPT_GQA_OK : OPT_GQA_ERR_CUDA;
+    // launched while the preceding grid drains; the kernel waits for it before it touches memory
+    return launch_dependent(cache_append_kernel, dim3((unsigned)blocks), dim3(threads), 0, stream,
+                            static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
+                            static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), slot_mapping, total, Hkv,
+                            row_vecs, bs);
 }
 
 }  // namespace optgqa
