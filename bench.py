@@ -6,6 +6,12 @@ cache_append of the step's new tokens -> paged GQA-ALiBi decode over context
 partitions -> log-sum-exp reduce.  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config 3] [--impl ours|reference]
+                  [--only step|prefill|projection]
+
+--steps / --warmup size the timed region behind `value`.  The legs that explain it have sample counts of their
+own, whatever --steps says: the decode kernel's launch duration comes from KERNEL_TIMING_STEPS further steps
+(event brackets around back-to-back launches), the end-to-end number from E2E_STEPS steps through host buffers,
+the read-only ceiling of the data path from a streaming probe over 1 GiB.
 
 N > 1 is launched with torch.distributed.run; the path shards by sequence with no
 data-path collective (every rank runs its own batch of the same shape), so the
@@ -34,6 +40,12 @@ DEFAULT_PARTITION = {2: 256, 3: 512, 4: 512}
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised
 # under profiles/ (None until a capture of that workload exists).
 NCU_TRAFFIC_BYTES = {3: 378_693_376 + 3_752_704}   # profiles/decode_stream_cfg3.md
+KERNEL_TIMING_STEPS = 512   # steps of the kernel-timing region (a bracket every EVENT_EVERY-th step)
+E2E_STEPS = 200             # steps of the end-to-end leg
+READ_PROBE_BYTES = 1 << 30  # bytes streamed by the read-only ceiling probe per launch
+DTYPE = "bf16 operands, f32 accumulate"
+KERNEL_FAMILY = ("tensor-core tile kernels: 2-D TMA tiles into per-warp rings, mma.sync m16n8k16 with the query group "
+                 "as one tile side, fp32 online softmax")
 
 
 # ----------------------------------------------------------------------------- distributed plumbing
@@ -79,8 +91,9 @@ _REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown"
 class ClockSampler(threading.Thread):
     """Samples SM clock and clock-event reasons of one GPU while the timed region runs (read-only NVML)."""
 
-    def __init__(self, device_index: int, period_s: float = 0.01):
+    def __init__(self, device_index: int, period_s: float = 0.002):
         super().__init__(daemon=True)
+        self.device_index = device_index
         self.period = period_s
         self.samples, self.reasons, self.sm_max = [], set(), None
         self._halt = threading.Event()
@@ -114,6 +127,14 @@ class ClockSampler(threading.Thread):
 
     def run(self):
         if self._h is None:
+            # no NVML binding: read-only nvidia-smi queries while the timed legs run
+            while not self._halt.is_set():
+                one = self._smi_query()
+                if one is not None:
+                    self.samples.append(one[0])
+                    self.sm_max = one[1]
+                    self.reasons.update(one[2])
+                self._halt.wait(0.05)
             return
         while not self._halt.is_set():
             try:
@@ -125,21 +146,24 @@ class ClockSampler(threading.Thread):
     def stop(self) -> dict:
         self._halt.set()
         self.join(timeout=2.0)
-        if self._h is None or not self.samples:
-            return self._smi_fallback()
-        s = sorted(self.samples)
-        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.sm_max, "reasons": sorted(self.reasons),
-                "samples": len(s)}
-
-    @staticmethod
-    def _smi_fallback() -> dict:
-        try:
-            out = subprocess.run(["nvidia-smi", "--query-gpu=clocks.sm,clocks.max.sm", "--format=csv,noheader,nounits"],
-                                 capture_output=True, text=True, timeout=10).stdout.strip().splitlines()[0]
-            a, b = [int(x) for x in out.split(",")]
-            return {"sm_mhz": a, "sm_max_mhz": b, "reasons": [], "samples": 1, "note": "one nvidia-smi sample after the run"}
-        except Exception:
+        if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_min_mhz": s[0], "sm_max_mhz": self.sm_max, "reasons": sorted(self.reasons),
+                "samples": len(s), "source": "nvml" if self._h is not None else "nvidia-smi"}
+
+    def _smi_query(self):
+        fields = ["clocks.sm", "clocks.max.sm", "clocks_event_reasons.hw_slowdown",
+                  "clocks_event_reasons.hw_thermal_slowdown", "clocks_event_reasons.sw_thermal_slowdown",
+                  "clocks_event_reasons.sw_power_cap"]
+        try:
+            out = subprocess.run(["nvidia-smi", "-i", str(self.device_index), "--query-gpu=" + ",".join(fields),
+                                  "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=10)
+            cells = [c.strip() for c in out.stdout.strip().splitlines()[0].split(",")]
+            reasons = [f.split(".")[1] for f, c in zip(fields[2:], cells[2:]) if c.lower().startswith("active")]
+            return int(cells[0]), int(cells[1]), reasons
+        except Exception:
+            return None
 
 
 # ----------------------------------------------------------------------------- workload on the device
@@ -166,6 +190,7 @@ class DeviceBatch:
         self.maxP = max(1, (int(wl.context_lens.max()) + partition_size - 1) // partition_size) if partition_size else 1
         ws = binding.workspace_bytes(wl.B, wl.Hq, wl.D, self.maxP) if partition_size else 0
         self.workspace = torch.empty(max(ws, 16), dtype=torch.uint8, device=device)
+        self.ws_bytes = int(self.workspace.numel())
         npart = wl.B * wl.Hq * self.maxP
         self.partial_out = self.workspace[: npart * wl.D * 4].view(torch.float32)
         self.partial_lse = self.workspace[npart * wl.D * 4: npart * (wl.D + 1) * 4].view(torch.float32) if ws else None
@@ -188,12 +213,8 @@ class DeviceBatch:
         if self.balanced:
             return (self.q.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(), self.tables.data_ptr(),
                     wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D,
-                    wl.bs, wl.num_blocks, self.P, self.workspace.data_ptr(), self.maxP, self.dt, stream)
-        return (self.out.data_ptr(), self.q.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(),
-                self.tables.data_ptr(), wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B,
-                wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, self.P,
-                self.partial_out.data_ptr() if self.P else None, self.partial_lse.data_ptr() if self.P else None,
-                self.maxP, self.dt, stream)
+                    wl.bs, wl.num_blocks, self.P, self.workspace.data_ptr(), self.ws_bytes, self.maxP, self.dt, stream)
+        return self.args_decode_plain(i, stream)
 
     def args_decode_plain(self, i, stream):
         """opt_gqa_paged_attention_decode: single pass (P = 0) or one partial per partition."""
@@ -207,8 +228,8 @@ class DeviceBatch:
     def args_reduce(self, stream):
         wl = self.wl
         if self.balanced:
-            return (self.out.data_ptr(), self.workspace.data_ptr(), self.lens.data_ptr(), wl.B, wl.Hq, wl.Hkv, wl.D,
-                    self.P, self.maxP, self.dt, stream)
+            return (self.out.data_ptr(), self.workspace.data_ptr(), self.ws_bytes, self.lens.data_ptr(), wl.B, wl.Hq,
+                    wl.Hkv, wl.D, self.P, self.maxP, self.dt, stream)
         return (self.out.data_ptr(), self.partial_out.data_ptr(), self.partial_lse.data_ptr(), self.lens.data_ptr(),
                 wl.B, wl.Hq, wl.D, self.P, self.maxP, self.dt, stream)
 
@@ -217,8 +238,8 @@ class DeviceBatch:
         return (self.out.data_ptr(), self.q.data_ptr(), self.k_new.data_ptr(), self.v_new.data_ptr(),
                 self.slots.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(), self.tables.data_ptr(),
                 wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D,
-                wl.bs, wl.num_blocks, self.P, self.workspace.data_ptr() if self.P else None, self.maxP, self.dt,
-                stream)
+                wl.bs, wl.num_blocks, self.P, self.workspace.data_ptr() if self.P else None,
+                self.ws_bytes if self.P else 0, self.maxP, self.dt, stream)
 
     def algorithmic_bytes(self) -> int:
         """Bytes one decode launch must move: every K and V element of every context once, q, out, table entries."""
@@ -290,12 +311,14 @@ class PrefillBatch:
 
 
 def measured_tensor_peak():
+    """(sustained, burst, kind) dense bf16 TFLOP/s: the measured cuBLAS figures, else the earlier pool measurement."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+            d = json.load(f)
+        return float(d["bf16_tflops_sustained"]), float(d["bf16_tflops"]), "measured"
     except Exception:
-        return 1400.0, "fallback (sustained)"
+        return 1400.0, 1590.0, "fallback"
 
 
 def prefill_report(dev, steps: int, warmup: int) -> dict:
@@ -305,18 +328,19 @@ def prefill_report(dev, steps: int, warmup: int) -> dict:
     wl = W.make_config(5)
     pb = PrefillBatch(wl, dev)
     step_ms, pf_ms = pb.run(steps, warmup)
-    peak, kind = measured_tensor_peak()
+    sustained, burst, kind = measured_tensor_peak()
     tf = pb.flops() / (pf_ms * 1e-3) / 1e12
     return {"new_tokens_per_s": wl.T / (step_ms * 1e-3), "ms_per_step": step_ms, "prefill_us": pf_ms * 1e3,
-            "prefill_TFLOPs": tf, "frac_of_bf16_peak": tf / peak, "peak": peak, "peak_kind": f"of {kind}",
-            "flop_per_launch": pb.flops(), "bound": "tensor"}
+            "prefill_TFLOPs": tf, "frac_of_bf16_peak": tf / sustained, "peak": sustained,
+            "peak_kind": f"of {kind} (sustained cuBLAS bf16)", "frac_of_bf16_burst_peak": tf / burst, "burst_peak": burst,
+            "launches_timed": steps, "flop_per_launch": pb.flops(), "bound": "tensor"}
 
 
 PROJECTION_SHAPES = (("width4096_32q4kv_T8", 8, 4096, 32, 4, 128), ("width8192_64q8kv_T8", 8, 8192, 64, 8, 128),
                      ("width8192_64q8kv_T16", 16, 8192, 64, 8, 128))
 
 
-def projection_report(dev, only=None) -> dict:
+def projection_report(dev) -> dict:
     """Side measurement of the 4-bit Q/K/V projection that precedes the step: one launch per layer-sized weight
     matrix, rotating through enough distinct matrices to exceed L2.  The launches are shorter than a foreign call
     from Python, so they are timed as one captured graph."""
@@ -331,8 +355,6 @@ def projection_report(dev, only=None) -> dict:
     out = {}
     side = torch.cuda.Stream()
     for name, T, K, Hq, Hkv, D in PROJECTION_SHAPES:
-        if only is not None and name != only:
-            continue
         N, gs = (Hq + 2 * Hkv) * D, 128
         p = W.make_int4_projection(11, T, K, N, gs)
         nbytes = binding.int4_packed_bytes(K, N, gs)
@@ -455,10 +477,17 @@ def _step_fns(batch: DeviceBatch, stream):
 
 def step_launches(batch: DeviceBatch) -> int:
     """Kernels one opt_gqa_decode_step call launches: decode + reduce on the split path, plus the separate append
-    unless the decode kernel stores the new tokens itself (bf16 split with at most 1024 (sequence, KV head) streams)."""
+    unless the decode kernel stores the new tokens itself (bf16 split with at most 1024 (sequence, KV head) streams);
+    one launch in all where the library runs a bf16 step of short contexts as a single pass (the rule of api.cu)."""
+    import torch
+
     if batch.P == 0:
         return 2
-    fused = batch.balanced and batch.wl.B * batch.wl.Hkv <= 1024
+    streams, bound = batch.wl.B * batch.wl.Hkv, batch.maxP * batch.P
+    sms = torch.cuda.get_device_properties(batch.dev).multi_processor_count
+    if batch.balanced and bound <= 2048 and 2 * streams >= 3 * sms and streams <= 4 * sms:
+        return 1
+    fused = batch.balanced and streams <= 1024
     return 2 if fused else 3
 
 
@@ -495,7 +524,8 @@ def run_kernel_timing(batch: DeviceBatch, steps: int, warmup: int):
     DECODE_BATCH is the duration of one launch in a pipelined stream: the launches are chained by programmatic
     dependent launch exactly as append -> decode is in a step, so the bracket's own event and launch gaps are
     paid once per DECODE_BATCH launches); odd samples bracket a single launch (which also pays those gaps).
-    Returns (ms per launch from the batched brackets, ms per launch from the single brackets, launches).
+    Returns (stats of ms per launch from the batched brackets, the same from the single brackets, launches);
+    stats = {"mean", "median", "min", "brackets", "launches"}.
     """
     import torch
 
@@ -526,8 +556,45 @@ def run_kernel_timing(batch: DeviceBatch, steps: int, warmup: int):
     barrier()
     batched = [evs[i][0].elapsed_time(evs[i][1]) / DECODE_BATCH for i in samples if (i // EVENT_EVERY) % 2 == 0]
     single = [evs[i][0].elapsed_time(evs[i][1]) for i in samples if (i // EVENT_EVERY) % 2 == 1]
-    mean = lambda v: sum(v) / len(v) if v else None
-    return mean(batched), mean(single), launches
+    def stats(v, per):
+        if not v:
+            return None
+        w = sorted(v)
+        return {"mean": sum(w) / len(w), "median": w[len(w) // 2], "min": w[0], "brackets": len(w),
+                "launches": len(w) * per}
+
+    return stats(batched, DECODE_BATCH), stats(single, 1), launches
+
+
+def read_only_ceiling(dev, stream) -> dict:
+    """GB/s of the decode kernels' data path with no arithmetic attached: opt_gqa_debug_read_stream over 1 GiB,
+    CUDA events on the launching stream, 3 warm-up and 10 timed launches (the buffer is 8x the L2)."""
+    import torch
+
+    from paper_2505_02351_b200 import binding
+
+    lib = binding.load()
+    src = torch.empty(READ_PROBE_BYTES, dtype=torch.uint8, device=dev)
+    src.view(torch.int32).fill_(0x3f803f80)
+    chk = torch.zeros(1, dtype=torch.int32, device=dev)
+    a = (src.data_ptr(), READ_PROBE_BYTES, chk.data_ptr(), stream.cuda_stream)
+    for _ in range(3):
+        check(lib.opt_gqa_debug_read_stream(*a), "read_stream")
+    torch.cuda.synchronize()
+    spans = []
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        check(lib.opt_gqa_debug_read_stream(*a), "read_stream")
+        e1.record(stream)
+        torch.cuda.synchronize()
+        spans.append(e0.elapsed_time(e1))
+    spans.sort()
+    del src
+    torch.cuda.empty_cache()
+    gbs = lambda ms: READ_PROBE_BYTES / (ms * 1e-3) / 1e9
+    return {"median": gbs(spans[len(spans) // 2]), "best": gbs(spans[0]), "launches": len(spans),
+            "bytes_per_launch": READ_PROBE_BYTES}
 
 
 def run_e2e(batch: DeviceBatch, steps: int, warmup: int):
@@ -553,7 +620,7 @@ def run_e2e(batch: DeviceBatch, steps: int, warmup: int):
     a_host = [(hout.data_ptr(), hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), hs.data_ptr(), ht.data_ptr(), hl.data_ptr(),
                staging.data_ptr(), batch.k_pools[i].data_ptr(), batch.v_pools[i].data_ptr(), wl.max_blocks,
                batch.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, batch.P, ws_ptr,
-               batch.maxP, batch.dt, sh) for i in range(R)]
+               batch.ws_bytes if batch.P else 0, batch.maxP, batch.dt, sh) for i in range(R)]
 
     def step(i):
         check(lib.opt_gqa_decode_step_host(*a_host[i % R]), "decode_step_host")
@@ -616,7 +683,18 @@ def cpu_baseline(wl, budget_s: float = 12.0) -> dict:
                       f"{best:.3f} s per pass"}
 
 
-def run_reference(args, wl, rank: int):
+def workload_config(wl, P: int, world: int, copies: int) -> dict:
+    """The `config` object of the result line; both arms (ours and the CPU reference) print the same one."""
+    return {"workload": wl.name, "batch_per_gpu": wl.B, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.D,
+            "block_size": wl.bs, "storage_dtype": wl.dtype, "partition_size": P,
+            "context_tokens_per_gpu": int(wl.context_lens.sum()),
+            "parallelism": f"dp{world} (by sequence, no collective)",
+            "step": "append of one token per sequence + paged GQA-ALiBi decode over context partitions + merge",
+            "l2": f"each step reads {wl.kv_bytes() / 1e6:.0f} MB of K/V (> 126 MB L2); on the GPU {copies} distinct "
+                  f"copies of the pool are rotated between steps"}
+
+
+def run_reference(args, wl, P: int, rank: int):
     """--impl reference: the oracle as it stands, on the host cores; each step a bounded sample."""
     fn, B = oracle_step_fn(wl)
     steps = args.steps if args.steps is not None else 5
@@ -636,8 +714,7 @@ def run_reference(args, wl, rank: int):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "batch": wl.B, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.D,
-                   "block_size": wl.bs, "storage_dtype": wl.dtype, "sample": sample},
+        "config": workload_config(wl, P, args.gpus, COPIES),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": omp_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -655,6 +732,10 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+COPIES = 4          # distinct KV pool copies rotated between steps
+PROFILE_COPIES = 2  # with --only: a footprint small enough for a profiler's capture
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -664,16 +745,9 @@ def main():
     ap.add_argument("--config", type=int, default=3, choices=[2, 3, 4],
                     help="named workload (1-based): 3 = long-sequence decode, the headline")
     ap.add_argument("--partition", type=int, default=None, help="context partition size (default: the workload's)")
-    ap.add_argument("--copies", type=int, default=4, help="distinct KV pool copies rotated between steps")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
-    ap.add_argument("--no-extra", action="store_true", help="skip the short side measurements of the other workloads")
-    ap.add_argument("--prefill-only", action="store_true",
-                    help="run only the chunked-prefill side measurement and print its report (profiling runs)")
-    ap.add_argument("--projection-only", action="store_true",
-                    help="run only the 4-bit Q/K/V projection side measurement and print its report (profiling runs)")
-    ap.add_argument("--projection-shape", default=None, choices=[s[0] for s in PROJECTION_SHAPES],
-                    help="with --projection-only: measure this shape alone")
+    ap.add_argument("--only", choices=["step", "prefill", "projection"], default=None,
+                    help="run one part alone on a small footprint and print its report: the decode step's two timed "
+                         "regions, the chunked-prefill workload, or the 4-bit projection (for profiler captures)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
 
@@ -683,7 +757,7 @@ def main():
         if rank != 0:
             return
         wl = W.make_config(args.config)
-        run_reference(args, wl, rank)
+        run_reference(args, wl, wl.partition_size or DEFAULT_PARTITION[args.config], rank)
         return
 
     import torch
@@ -699,93 +773,104 @@ def main():
         import torch.distributed as dist
 
         dist.init_process_group("nccl", device_id=dev)
-    if args.prefill_only:
+    if args.only == "prefill":
         if rank == 0:
             print(json.dumps(prefill_report(dev, args.steps or 20, max(3, args.warmup or 3))), flush=True)
         return
-    if args.projection_only:
+    if args.only == "projection":
         if rank == 0:
-            print(json.dumps(projection_report(dev, args.projection_shape)), flush=True)
+            print(json.dumps(projection_report(dev)), flush=True)
         return
     steps = args.steps if args.steps is not None else 4000
     warmup = max(3, args.warmup if args.warmup is not None else 50)
+    copies = PROFILE_COPIES if args.only else COPIES
 
     wl = W.make_config(args.config, seed_offset=1000 * rank)
     P = args.partition if args.partition is not None else (wl.partition_size or DEFAULT_PARTITION[args.config])
-    batch = DeviceBatch(wl, P, args.copies, dev)
-    pool_bytes = sum(t.numel() * t.element_size() for t in batch.k_pools + batch.v_pools)
+    batch = DeviceBatch(wl, P, copies, dev)
 
     sampler = ClockSampler(local_rank)
     sampler.start()
     total_ms, launches = run_timed(batch, steps, warmup)
-    dec_ms, dec_single_ms, launches2 = run_kernel_timing(batch, min(steps, 1024), 8)
+    kt_steps = steps if args.only else KERNEL_TIMING_STEPS
+    dec, dec_single, launches2 = run_kernel_timing(batch, kt_steps, 8)
     launches += launches2
-    clocks = sampler.stop()
-    status = binding.device_status()
-    if status != 0:
-        raise SystemExit(f"device status {status}: {binding.status_string(status)}")
     total_ms = max_over_ranks(total_ms, str(dev))
     tokens_all = sum_over_ranks(float(wl.B), str(dev))
     value = tokens_all * steps / (total_ms * 1e-3)
 
-    e2e_steps = min(steps, 500)
-    if args.no_e2e:
-        e2e_s, h2d, d2h = float("nan"), 0, 0
+    if args.only:
+        e2e = None
+        ceiling = None
     else:
-        e2e_s, h2d, d2h, _ = run_e2e(batch, e2e_steps, 10)
+        e2e_s, h2d, d2h, _ = run_e2e(batch, E2E_STEPS, 10)
         e2e_s = max_over_ranks(e2e_s, str(dev))
-    e2e_value = tokens_all * e2e_steps / e2e_s
+        e2e = {"value": tokens_all * E2E_STEPS / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": E2E_STEPS, "us_per_step": e2e_s / E2E_STEPS * 1e6,
+               "api": "opt_gqa_decode_step_host (pinned host q/k_new/v_new/slots/tables/lens in, out back, "
+                      "stream synchronised per step)"}
+        e2e["frac_of_value"] = e2e["value"] / value
+        ceiling = read_only_ceiling(dev, torch.cuda.current_stream())
+    clocks = sampler.stop()
+    status = binding.device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status}: {binding.status_string(status)}")
 
     peak, peak_kind = measured_peak()
     alg = batch.algorithmic_bytes()
-    achieved = alg / (dec_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (balanced split)" if batch.balanced else "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(args.config),
-                "algorithmic_bytes_per_launch": alg, "kernel_us": dec_ms * 1e3,
-                "kernel_us_single_launch_bracket": None if dec_single_ms is None else dec_single_ms * 1e3,
+    achieved = alg / (dec["mean"] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (balanced split)" if batch.balanced else "decode_kernel",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                "algorithmic_bytes_per_launch": alg, "kernel_us": dec["mean"] * 1e3,
+                "kernel_us_median": dec["median"] * 1e3, "kernel_us_min": dec["min"] * 1e3,
+                "launches_timed": dec["launches"], "brackets": dec["brackets"],
+                "kernel_us_single_launch_bracket": None if dec_single is None else dec_single["mean"] * 1e3,
                 "timing": f"CUDA events around {DECODE_BATCH} back-to-back decode launches on successive pool copies, "
-                          f"every {2 * EVENT_EVERY}th step of a second timed region; span / {DECODE_BATCH}",
+                          f"every {2 * EVENT_EVERY}th step of a second timed region of {kt_steps} steps; span / {DECODE_BATCH}",
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+    if ceiling is not None:
+        roofline["read_only_ceiling_gbs"] = ceiling["median"]
+        roofline["read_only_ceiling_best_gbs"] = ceiling["best"]
+        roofline["frac_of_read_ceiling"] = achieved / ceiling["median"]
+        roofline["read_only_ceiling"] = (f"opt_gqa_debug_read_stream over {READ_PROBE_BYTES >> 20} MiB, same rings and grid "
+                                         f"as the decode kernel, no arithmetic; median of {ceiling['launches']} launches")
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "batch_per_gpu": wl.B, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.D,
-                   "block_size": wl.bs, "storage_dtype": wl.dtype, "partition_size": P,
-                   "context_tokens_per_gpu": int(wl.context_lens.sum()), "parallelism": f"dp{world} (by sequence, no collective)",
-                   "step": "opt_gqa_decode_step: append of one token per sequence (stored by the decode kernel) + decode + reduce",
-                   "l2": f"{args.copies} distinct KV pool copies ({pool_bytes / 1e9:.2f} GB) rotated between steps; "
-                         f"each step reads {wl.kv_bytes() / 1e6:.0f} MB (> 126 MB L2)"},
+        "dtype": DTYPE, "data": "synthetic",
+        "config": workload_config(wl, P, world, copies),
+        "kernel_family": KERNEL_FAMILY,
+        "api": "opt_gqa_decode_step (new tokens stored by the decode kernel, balanced split, merge)",
         "hbm_tbs_step": alg * tokens_all / wl.B / (total_ms / steps * 1e-3) / 1e12,
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "api": "opt_gqa_decode_step_host (pinned host q/k_new/v_new/slots/tables/lens in, out back, sync per step)"},
         "gpu_launches": launches,
         "roofline": roofline,
     }
+    if e2e is not None:
+        line["e2e"] = e2e
 
-    if rank == 0 and world == 1 and not args.no_extra:
+    if rank == 0 and world == 1 and not args.only:
         extra = {}
         for cfg in (2, 4):
             if cfg == args.config:
                 continue
             w2 = W.make_config(cfg)
-            b2 = DeviceBatch(w2, w2.partition_size or DEFAULT_PARTITION[cfg], args.copies, dev)
+            b2 = DeviceBatch(w2, w2.partition_size or DEFAULT_PARTITION[cfg], COPIES, dev)
             t_ms, _ = run_timed(b2, 1000, 20)
-            d_ms, _, _ = run_kernel_timing(b2, 256, 8)
+            d2, _, _ = run_kernel_timing(b2, 256, 8)
             a2 = b2.algorithmic_bytes()
             extra[w2.name] = {"tokens_per_s": w2.B * 1000 / (t_ms * 1e-3), "ms_per_step": t_ms / 1000,
-                              "decode_us": d_ms * 1e3, "decode_GBs": a2 / (d_ms * 1e-3) / 1e9,
-                              "frac_of_peak": a2 / (d_ms * 1e-3) / 1e9 / peak, "partition_size": b2.P}
+                              "decode_us": d2["mean"] * 1e3, "decode_GBs": a2 / (d2["mean"] * 1e-3) / 1e9,
+                              "frac_of_peak": a2 / (d2["mean"] * 1e-3) / 1e9 / peak, "partition_size": b2.P,
+                              "launches_timed": d2["launches"]}
             del b2, w2
             torch.cuda.empty_cache()
         extra["other_decode_entry_points"] = entry_point_report(dev, peak)
         extra[W.CONFIG_NAMES[5]] = prefill_report(dev, 20, 3)
         extra["int4_qkv_projection"] = projection_report(dev)
         line["other_workloads"] = extra
-
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl)
     if world > 1:
         import torch.distributed as dist

@@ -14,7 +14,22 @@
  *    documented as HOST.  The library allocates nothing and keeps no pointer after
  *    the call returns; calls only enqueue work on `stream` (a cudaStream_t passed as
  *    void*, NULL = the default stream) and return.  The caller keeps every buffer
- *    alive until that work has finished.
+ *    alive until that work has finished.  `stream` must belong to the current device.
+ *  - State of the library, all of it per device: one status word in device memory
+ *    (opt_gqa_device_status), the fixed scratch array of the _no_alloc entry point, and
+ *    host-side caches of symbol addresses and kernel attributes filled by the first call
+ *    on a device (make that call outside stream capture).  The caches are atomics: calls
+ *    from several host threads are safe, also when they are the first ones.
+ *  - Ordering inside a stream: the kernels are launched with programmatic stream
+ *    serialisation and wait for the preceding kernel of the stream before they read
+ *    anything it may write (q, k_new, v_new, the cache, the partials) or overwrite
+ *    anything it may read (out, the workspace).  Two index arrays are the exception:
+ *    block_tables and context_lens are read BEFORE that wait (the split of the work is
+ *    computed from them while the preceding kernel drains).  They must therefore not be
+ *    produced by a kernel that signals its dependents early (griddepcontrol
+ *    .launch_dependents / cudaTriggerProgrammaticLaunchCompletion); no kernel of this
+ *    library writes them except the gather of opt_gqa_decode_step_host, which does not
+ *    signal early.  Ordinary producers (copies, kernels without that signal) are fine.
  *  - dtype: OPT_GQA_FP32 (0) or OPT_GQA_BF16 (1).  q, k_new/v_new, the cache and out
  *    share it.  Slopes, scale, partials are always fp32.  All arithmetic is fp32;
  *    results are rounded once (to nearest even) when stored.
@@ -134,8 +149,10 @@ int opt_gqa_paged_attention_decode_simt(void* out, const void* q, const void* k_
  * opt_gqa_paged_attention_reduce_balanced (same B, Hq, Hkv, D, partition_size,
  * max_partitions, same workspace, later on the same stream) merges them into out.
  *
- *   workspace     opt_gqa_workspace_bytes(B, Hq, D, max_partitions) bytes, 16-byte aligned;
- *                 contents need no initialisation and are overwritten
+ *   workspace     device memory, 16-byte aligned; contents need no initialisation and are overwritten
+ *   workspace_bytes  HOST value: the size of `workspace`; OPT_GQA_ERR_SHAPE if it is below what the
+ *                 split of these sizes needs (opt_gqa_workspace_bytes(B, Hq, D, max_partitions) always
+ *                 suffices)
  *   partition_size  P > 0, a multiple of 16;  max_partitions >= ceil(max_s n_s / P)
  * Other arguments as in opt_gqa_paged_attention_decode.  dtype must be OPT_GQA_BF16.
  */
@@ -143,8 +160,8 @@ int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, 
                                             const int32_t* block_tables, int max_blocks_per_seq,
                                             const int32_t* context_lens, const float* alibi_slopes, float scale,
                                             int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
-                                            int partition_size, void* workspace, int max_partitions, int dtype,
-                                            void* stream);
+                                            int partition_size, void* workspace, size_t workspace_bytes,
+                                            int max_partitions, int dtype, void* stream);
 
 /*
  * Log-sum-exp merge of the pieces written by opt_gqa_paged_attention_decode_balanced (the
@@ -152,9 +169,9 @@ int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, 
  *     out = sum_c e^{lse_c} o_c / sum_c e^{lse_c}   over the pieces c of the row's sequence and KV head.
  * out [B, Hq, D] in `dtype`; n_s == 0 gives zero rows.
  */
-int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B,
-                                            int Hq, int Hkv, int D, int partition_size, int max_partitions,
-                                            int dtype, void* stream);
+int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, size_t workspace_bytes,
+                                            const int32_t* context_lens, int B, int Hq, int Hkv, int D,
+                                            int partition_size, int max_partitions, int dtype, void* stream);
 
 /*
  * Merge of the partitions' results (the paragraph before Eq. 1: each partition's
@@ -189,6 +206,7 @@ int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const fl
  *    what a previous call left in it is never read.
  *  - The first call on each device looks up the array's device address (a runtime call
  *    made with that device current); make that first call outside any stream capture.
+ *    The address belongs to the CURRENT device: `stream` must be a stream of that device.
  */
 int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q, const void* k_cache, const void* v_cache,
                                             const int32_t* block_tables, int max_blocks_per_seq,
@@ -245,7 +263,8 @@ int opt_gqa_paged_attention_decode_local(void* out, const void* q, const void* k
                                          const int32_t* block_tables, int max_blocks_per_seq,
                                          const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
                                          int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                                         void* workspace, int max_partitions, int window, int dtype, void* stream);
+                                         void* workspace, size_t workspace_bytes, int max_partitions, int window,
+                                         int dtype, void* stream);
 
 int opt_gqa_paged_attention_prefill_local(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
                                           int max_q_len, const void* k_cache, const void* v_cache,
@@ -314,11 +333,17 @@ int opt_gqa_qkv_project_int4(void* q_out, void* k_out, void* v_out, void* k_cach
  * into C_K, C_V" to "Compute context attention with caches": cache_append of the
  * B new tokens (k_new, v_new [B, Hkv, D], slot_mapping [B]), then decode, then --
  * when partition_size > 0 -- the reduce, all enqueued on `stream` by one call.
- * workspace: opt_gqa_workspace_bytes(B, Hq, D, max_partitions) bytes of device
- * memory, 16-byte aligned; may be NULL when partition_size is 0.  bf16 caches take
+ * workspace: workspace_bytes (a HOST value) bytes of device memory, 16-byte aligned;
+ * opt_gqa_workspace_bytes(B, Hq, D, max_partitions) suffices, less than the step needs
+ * is refused with OPT_GQA_ERR_SHAPE before anything is enqueued; may be NULL (and 0)
+ * when partition_size is 0.  bf16 caches take
  * the balanced split (decode_balanced + reduce_balanced), fp32 caches one partial
  * per partition (partial_out followed by partial_lse at the start of workspace).
  * Other arguments as in the calls it chains.  out [B, Hq, D] is always written.
+ * A bf16 step whose contexts are all short (max_partitions * partition_size <= 2048) and whose (sequence, KV
+ * head) streams number between 1.5 and 4 times the GPU's multiprocessors runs as a single launch: one CTA per
+ * stream walks the whole context, stores the stream's new token itself and writes out (the result is the same;
+ * the workspace is not touched).
  * On the bf16 split path with at most 1024 (sequence, KV head) streams no separate append kernel
  * runs: the decode kernel stores sequence s's new token to slot_mapping[s] itself, just before it
  * fetches the tile that holds position context_lens[s] - 1 (a sequence with context_lens 0 has no
@@ -328,7 +353,8 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
                         const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,
                         int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,
                         float scale, int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
-                        int partition_size, void* workspace, int max_partitions, int dtype, void* stream);
+                        int partition_size, void* workspace, size_t workspace_bytes, int max_partitions, int dtype,
+                        void* stream);
 
 /*
  * The same step for a caller whose per-step tensors live in HOST memory (pinned,
@@ -349,7 +375,7 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
                              const int32_t* context_lens_host, void* staging, void* k_cache, void* v_cache,
                              int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
                              int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
-                             int max_partitions, int dtype, void* stream);
+                             size_t workspace_bytes, int max_partitions, int dtype, void* stream);
 
 /* Device bytes opt_gqa_decode_step_host needs in `staging`.  Host arithmetic; 0 for bad arguments. */
 size_t opt_gqa_step_staging_bytes(int B, int Hq, int Hkv, int D, int max_blocks_per_seq, int dtype);
@@ -362,6 +388,26 @@ size_t opt_gqa_step_staging_bytes(int B, int Hq, int Hkv, int D, int max_blocks_
  * partitioning step; pure host arithmetic.)  Returns 0 for non-positive arguments.
  */
 size_t opt_gqa_workspace_bytes(int B, int Hq, int D, int max_partitions);
+
+/*
+ * Diagnostics for the bounded waits (no counterpart in the paper).  Every wait of a kernel on an
+ * mbarrier gives up after about 2^28 SM clocks, records OPT_GQA_ERR_TIMEOUT in the status word and
+ * lets the kernel return.  This call makes exactly that happen, so that a host's handling of the
+ * status can be tested without a fault or a hang: it launches one warp on `stream` that waits, with
+ * a limit of limit_cycles SM clocks (1 .. 2^24; OPT_GQA_ERR_SHAPE otherwise), for bytes that nothing
+ * sends.  After the stream has drained opt_gqa_device_status() returns OPT_GQA_ERR_TIMEOUT once.
+ */
+int opt_gqa_debug_wait_timeout(long long limit_cycles, void* stream);
+
+/*
+ * Read-only streaming probe (diagnostics; no counterpart in the paper): streams `bytes` bytes from
+ * src through the same per-warp rings of bulk async copies, in the same grid shape, as the decode
+ * kernels, with no arithmetic attached -- the rate it reaches is the ceiling of that data path on
+ * this GPU.  bytes must be a multiple of 8192 and src 16-byte aligned.  A checksum (XOR of one
+ * 16-byte word per lane and chunk) is XOR-ed into *checksum (device memory), so that the reads
+ * cannot be optimised away; time the call with events on `stream`.
+ */
+int opt_gqa_debug_read_stream(const void* src, size_t bytes, unsigned* checksum, void* stream);
 
 /*
  * Reads and clears the device status word of the current device: 0, or

@@ -21,7 +21,7 @@ FP32, BF16 = 0, 1
 _DTYPE_CODE = {torch.float32: FP32, torch.bfloat16: BF16}
 
 _c = ctypes
-_vp, _i, _i64, _f = _c.c_void_p, _c.c_int, _c.c_int64, _c.c_float
+_vp, _i, _i64, _f, _sz = _c.c_void_p, _c.c_int, _c.c_int64, _c.c_float, _c.c_size_t
 
 SIGNATURES = {
     "opt_gqa_int4_packed_bytes": (ctypes.c_size_t, [_i, _i, _i]),
@@ -33,8 +33,8 @@ SIGNATURES = {
     "opt_gqa_paged_attention_decode_simt": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
                                                  _i, _vp, _vp, _i, _i, _vp]),
     "opt_gqa_paged_attention_decode_balanced": (_i, [_vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
-                                                     _i, _vp, _i, _i, _vp]),
-    "opt_gqa_paged_attention_reduce_balanced": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp]),
+                                                     _i, _vp, _sz, _i, _i, _vp]),
+    "opt_gqa_paged_attention_reduce_balanced": (_i, [_vp, _vp, _sz, _vp, _i, _i, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_decode_no_alloc": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i,
                                                      _i64, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_reduce": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
@@ -43,16 +43,18 @@ SIGNATURES = {
     "opt_gqa_paged_attention_prefill_mma": (_i, [_vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i,
                                                  _i, _i, _i64, _i, _vp]),
     "opt_gqa_paged_attention_decode_local": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
-                                                  _i, _vp, _i, _i, _i, _vp]),
+                                                  _i, _vp, _sz, _i, _i, _i, _vp]),
     "opt_gqa_paged_attention_prefill_local": (_i, [_vp, _vp, _vp, _i, _i, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i,
                                                    _i, _i, _i64, _i, _i, _vp]),
     "opt_gqa_prompt_attention": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _vp, _f, _i, _i, _i, _i, _i, _vp]),
     "opt_gqa_decode_step": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp, _f, _i, _i, _i, _i, _i, _i64,
-                                 _i, _vp, _i, _i, _vp]),
+                                 _i, _vp, _sz, _i, _i, _vp]),
     "opt_gqa_decode_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _f, _i, _i, _i, _i,
-                                      _i, _i64, _i, _vp, _i, _i, _vp]),
+                                      _i, _i64, _i, _vp, _sz, _i, _i, _vp]),
     "opt_gqa_step_staging_bytes": (_c.c_size_t, [_i, _i, _i, _i, _i, _i]),
     "opt_gqa_workspace_bytes": (_c.c_size_t, [_i, _i, _i, _i]),
+    "opt_gqa_debug_wait_timeout": (_i, [_c.c_longlong, _vp]),
+    "opt_gqa_debug_read_stream": (_i, [_vp, _sz, _vp, _vp]),
     "opt_gqa_device_status": (_i, []),
     "opt_gqa_status_string": (_c.c_char_p, [_i]),
 }
@@ -113,6 +115,22 @@ def device_status() -> int:
     return int(load().opt_gqa_device_status())
 
 
+def debug_wait_timeout(limit_cycles: int, stream=None) -> None:
+    """Launches one warp whose bounded wait runs out after `limit_cycles` SM clocks (sets the device status)."""
+    _check(load().opt_gqa_debug_wait_timeout(limit_cycles, _stream(stream)), "opt_gqa_debug_wait_timeout")
+
+
+def debug_read_stream(src, checksum, stream=None) -> None:
+    """Streams all of `src` through the decode kernels' data path with no arithmetic (read-bandwidth ceiling)."""
+    assert checksum.dtype == torch.int32 and checksum.numel() >= 1
+    _check(load().opt_gqa_debug_read_stream(_ptr(src), src.numel() * src.element_size(), _ptr(checksum),
+                                            _stream(stream)), "opt_gqa_debug_read_stream")
+
+
+def _nbytes(t: Optional[torch.Tensor]) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
 def cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, stream=None) -> None:
     T, Hkv, D = k_new.shape
     num_blocks, _, bs, _ = k_cache.shape
@@ -154,19 +172,18 @@ def paged_attention_decode_balanced(q, k_cache, v_cache, block_tables, context_l
     num_blocks, Hkv, bs, _ = k_cache.shape
     assert block_tables.dtype == torch.int32 and context_lens.dtype == torch.int32
     assert alibi_slopes is None or alibi_slopes.dtype == torch.float32
-    assert workspace.numel() * workspace.element_size() >= workspace_bytes(B, Hq, D, max_partitions)
     _check(load().opt_gqa_paged_attention_decode_balanced(
         _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables), block_tables.shape[1], _ptr(context_lens),
-        _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, _ptr(workspace), max_partitions,
-        _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_decode_balanced")
+        _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, _ptr(workspace), _nbytes(workspace),
+        max_partitions, _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_decode_balanced")
 
 
 def paged_attention_reduce_balanced(out, workspace, context_lens, Hkv: int, partition_size: int, max_partitions: int,
                                     stream=None) -> None:
     B, Hq, D = out.shape
     _check(load().opt_gqa_paged_attention_reduce_balanced(
-        _ptr(out), _ptr(workspace), _ptr(context_lens), B, Hq, Hkv, D, partition_size, max_partitions,
-        _DTYPE_CODE[out.dtype], _stream(stream)), "opt_gqa_paged_attention_reduce_balanced")
+        _ptr(out), _ptr(workspace), _nbytes(workspace), _ptr(context_lens), B, Hq, Hkv, D, partition_size,
+        max_partitions, _DTYPE_CODE[out.dtype], _stream(stream)), "opt_gqa_paged_attention_reduce_balanced")
 
 
 def paged_attention_decode_no_alloc(out, q, k_cache, v_cache, block_tables, context_lens, alibi_slopes, scale: float,
@@ -222,7 +239,8 @@ def paged_attention_decode_local(out, q, k_cache, v_cache, block_tables, context
     _check(load().opt_gqa_paged_attention_decode_local(
         _ptr(out), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_tables), block_tables.shape[1],
         _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, _ptr(workspace),
-        max_partitions, window, _DTYPE_CODE[q.dtype], _stream(stream)), "opt_gqa_paged_attention_decode_local")
+        _nbytes(workspace), max_partitions, window, _DTYPE_CODE[q.dtype], _stream(stream)),
+        "opt_gqa_paged_attention_decode_local")
 
 
 def paged_attention_prefill_local(out, q, q_start_loc, max_q_len: int, k_cache, v_cache, block_tables, context_lens,
@@ -283,8 +301,8 @@ def decode_step(out, q, k_new, v_new, slot_mapping, k_cache, v_cache, block_tabl
     _check(load().opt_gqa_decode_step(
         _ptr(out), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(slot_mapping), _ptr(k_cache), _ptr(v_cache),
         _ptr(block_tables), block_tables.shape[1], _ptr(context_lens), _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs,
-        num_blocks, partition_size, _ptr(workspace), max_partitions, _DTYPE_CODE[q.dtype], _stream(stream)),
-        "opt_gqa_decode_step")
+        num_blocks, partition_size, _ptr(workspace), _nbytes(workspace), max_partitions, _DTYPE_CODE[q.dtype],
+        _stream(stream)), "opt_gqa_decode_step")
 
 
 def _host_ptr(t: torch.Tensor) -> int:
@@ -303,5 +321,5 @@ def decode_step_host(out_host, q_host, k_new_host, v_new_host, slot_mapping_host
         _host_ptr(out_host), _host_ptr(q_host), _host_ptr(k_new_host), _host_ptr(v_new_host),
         _host_ptr(slot_mapping_host), _host_ptr(block_tables_host), _host_ptr(context_lens_host), _ptr(staging),
         _ptr(k_cache), _ptr(v_cache), block_tables_host.shape[1], _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs,
-        num_blocks, partition_size, _ptr(workspace), max_partitions, _DTYPE_CODE[q_host.dtype], _stream(stream)),
-        "opt_gqa_decode_step_host")
+        num_blocks, partition_size, _ptr(workspace), _nbytes(workspace), max_partitions, _DTYPE_CODE[q_host.dtype],
+        _stream(stream)), "opt_gqa_decode_step_host")

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libopt_gqa.so")
-SOURCES = ["api.cu", "cache_append.cu", "decode.cu", "decode_tc.cu", "decode_stream.cu", "reduce.cu", "prefill.cu", "prefill_umma.cu", "no_alloc.cu", "qkv_int4.cu"]
+SOURCES = ["api.cu", "cache_append.cu", "decode.cu", "decode_tc.cu", "decode_stream.cu", "reduce.cu", "prefill.cu", "prefill_umma.cu", "no_alloc.cu", "qkv_int4.cu", "diagnostics.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -31,7 +31,6 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "nvcc")
-    extra = os.environ.get("OPT_GQA_NVCC_FLAGS", "").split()   # e.g. -DOPT_GQA_TC_STAGES=3 for tuning sweeps
     objs = []
     build_dir = os.path.join(_PKG, "_build")
     os.makedirs(build_dir, exist_ok=True)
@@ -39,7 +38,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     for src in SOURCES:
         obj = os.path.join(build_dir, src.replace(".cu", ".o"))
         objs.append(obj)
-        cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))

@@ -1,5 +1,6 @@
 // extern "C" boundary of the Opt-GQA library: host-side argument checks, then one
-// launcher per operation.  Nothing here allocates or keeps caller pointers.
+// launcher per operation.  Nothing here allocates or keeps caller pointers; the only state of the
+// library is per device: a status word on the GPU and host-side caches of addresses and attributes.
 #include "common.cuh"
 
 namespace optgqa {
@@ -8,15 +9,17 @@ namespace optgqa {
 __device__ int g_device_status = 0;
 
 int* device_status_ptr() {
-    static int* ptrs[64] = {};
+    static std::atomic<int*> ptrs[kMaxDevices];
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ptrs[dev]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
-        ptrs[dev] = static_cast<int*>(p);
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    int* p = ptrs[dev].load(std::memory_order_acquire);
+    if (!p) {
+        void* v = nullptr;
+        if (cudaGetSymbolAddress(&v, g_device_status) != cudaSuccess || !v) return nullptr;
+        p = static_cast<int*>(v);
+        ptrs[dev].store(p, std::memory_order_release);
     }
-    return ptrs[dev];
+    return p;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -61,7 +64,7 @@ static int decode_checked(bool allow_tensor_cores, void* out, const void* q, con
     if (B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
     if (B == 0) return OPT_GQA_OK;
     if (!q || !k_cache || !v_cache || !block_tables || !context_lens) return OPT_GQA_ERR_NULL;
-    if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
+    if (num_blocks == 0 || max_blocks_per_seq == 0) return OPT_GQA_ERR_SHAPE;
     if (partition_size == 0) {
         if (!out) return OPT_GQA_ERR_NULL;
         if (!aligned16(out)) return OPT_GQA_ERR_ALIGN;
@@ -81,8 +84,8 @@ static int decode_checked(bool allow_tensor_cores, void* out, const void* q, con
                                 alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
                                 partial_lse, max_partitions, status, cs);
     return launch_decode(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
-                         scale, B, Hq, Hkv, D, bs, partition_size, partial_out, partial_lse, max_partitions, dtype,
-                         status, cs);
+                         scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out, partial_lse, max_partitions,
+                         dtype, status, cs);
 }
 
 int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache, const void* v_cache,
@@ -124,8 +127,9 @@ int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const fl
 static int decode_balanced_checked(const void* q, const void* k_cache, const void* v_cache,
                                    const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
                                    const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
-                                   int64_t num_blocks, int partition_size, void* workspace, int max_partitions,
-                                   int window, int dtype, void* stream, const FusedAppend* append = nullptr) {
+                                   int64_t num_blocks, int partition_size, void* workspace, size_t workspace_bytes,
+                                   int max_partitions, int window, int dtype, void* stream,
+                                   const FusedAppend* append = nullptr) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 || num_blocks < 0 || partition_size <= 0 ||
@@ -134,60 +138,63 @@ static int decode_balanced_checked(const void* q, const void* k_cache, const voi
     if (B > 65535 || Hkv > 65535 || max_partitions > 65535) return OPT_GQA_ERR_SHAPE;
     if (B == 0) return OPT_GQA_OK;
     if (!q || !k_cache || !v_cache || !block_tables || !context_lens || !workspace) return OPT_GQA_ERR_NULL;
-    if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
+    if (num_blocks == 0 || max_blocks_per_seq == 0) return OPT_GQA_ERR_SHAPE;
+    if (workspace_bytes < balanced_layout(B, Hq, Hkv, D, max_partitions).total) return OPT_GQA_ERR_SHAPE;
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(workspace)) return OPT_GQA_ERR_ALIGN;
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
     return launch_decode_stream(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
-                                scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, nullptr, nullptr, workspace,
-                                max_partitions, window, status, static_cast<cudaStream_t>(stream), append);
+                                scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, max_partitions, window,
+                                status, static_cast<cudaStream_t>(stream), append);
 }
 
 int opt_gqa_paged_attention_decode_balanced(const void* q, const void* k_cache, const void* v_cache,
                                             const int32_t* block_tables, int max_blocks_per_seq,
                                             const int32_t* context_lens, const float* alibi_slopes, float scale,
                                             int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
-                                            int partition_size, void* workspace, int max_partitions, int dtype,
-                                            void* stream) {
+                                            int partition_size, void* workspace, size_t workspace_bytes,
+                                            int max_partitions, int dtype, void* stream) {
     return decode_balanced_checked(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
-                                   scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, max_partitions, 0,
-                                   dtype, stream);
+                                   scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, workspace_bytes,
+                                   max_partitions, 0, dtype, stream);
 }
 
-static int reduce_balanced_checked(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq,
-                                   int Hkv, int D, int partition_size, int max_partitions, int window, int dtype,
-                                   void* stream) {
+static int reduce_balanced_checked(void* out, const void* workspace, size_t workspace_bytes,
+                                   const int32_t* context_lens, int B, int Hq, int Hkv, int D, int partition_size,
+                                   int max_partitions, int window, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128) || partition_size <= 0 ||
         partition_size % 16 != 0 || max_partitions <= 0 || window < 0)
         return OPT_GQA_ERR_SHAPE;
     if (B == 0) return OPT_GQA_OK;
     if (!out || !workspace || !context_lens) return OPT_GQA_ERR_NULL;
+    if (workspace_bytes < balanced_layout(B, Hq, Hkv, D, max_partitions).total) return OPT_GQA_ERR_SHAPE;
     if (!aligned16(out) || !aligned16(workspace)) return OPT_GQA_ERR_ALIGN;
     return launch_reduce_balanced(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, window,
                                   dtype, static_cast<cudaStream_t>(stream));
 }
 
-int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B,
-                                            int Hq, int Hkv, int D, int partition_size, int max_partitions,
-                                            int dtype, void* stream) {
-    return reduce_balanced_checked(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, 0, dtype,
-                                   stream);
+int opt_gqa_paged_attention_reduce_balanced(void* out, const void* workspace, size_t workspace_bytes,
+                                            const int32_t* context_lens, int B, int Hq, int Hkv, int D,
+                                            int partition_size, int max_partitions, int dtype, void* stream) {
+    return reduce_balanced_checked(out, workspace, workspace_bytes, context_lens, B, Hq, Hkv, D, partition_size,
+                                   max_partitions, 0, dtype, stream);
 }
 
 int opt_gqa_paged_attention_decode_local(void* out, const void* q, const void* k_cache, const void* v_cache,
                                          const int32_t* block_tables, int max_blocks_per_seq,
                                          const int32_t* context_lens, const float* alibi_slopes, float scale, int B,
                                          int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                                         void* workspace, int max_partitions, int window, int dtype, void* stream) {
+                                         void* workspace, size_t workspace_bytes, int max_partitions, int window,
+                                         int dtype, void* stream) {
     if (window <= 0) return OPT_GQA_ERR_SHAPE;
     if (B > 0 && !out) return OPT_GQA_ERR_NULL;
     int rc = decode_balanced_checked(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
-                                     scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, max_partitions,
-                                     window, dtype, stream);
+                                     scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, workspace_bytes,
+                                     max_partitions, window, dtype, stream);
     if (rc != OPT_GQA_OK || B == 0) return rc;
-    return reduce_balanced_checked(out, workspace, context_lens, B, Hq, Hkv, D, partition_size, max_partitions, window,
-                                   dtype, stream);
+    return reduce_balanced_checked(out, workspace, workspace_bytes, context_lens, B, Hq, Hkv, D, partition_size,
+                                   max_partitions, window, dtype, stream);
 }
 
 static int prefill_checked(bool allow_umma, int window, void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
@@ -265,17 +272,56 @@ int opt_gqa_prompt_attention(void* out, const void* q, const void* k, const void
                               status, static_cast<cudaStream_t>(stream));
 }
 
+// Bytes of `workspace` a decode step of these sizes uses: the balanced split's layout for bf16 caches, one
+// (D + 1)-float row per (sequence, head, partition) for fp32 caches, nothing for a single pass.
+static size_t step_workspace_need(int B, int Hq, int Hkv, int D, int partition_size, int max_partitions, int dtype) {
+    if (partition_size <= 0 || B <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || max_partitions <= 0) return 0;
+    if (dtype == OPT_GQA_BF16) return balanced_layout(B, Hq, Hkv, D, max_partitions).total;
+    return (size_t)B * Hq * max_partitions * ((size_t)D + 1) * 4;
+}
+
 // Streams (sequence x KV head) up to which opt_gqa_decode_step lets the streaming kernel store the new tokens.
 static constexpr long long kFusedAppendMaxStreams = 1024;
+
+// A bf16 step whose contexts are all short and whose (sequence, KV head) streams outnumber the SMs runs as ONE launch:
+// one CTA per stream walks its whole context, stores the stream's new token itself and writes out, so neither the
+// slot-mapped write nor the merge is a launch of its own (on such batches the two extra launches and the pieces'
+// round trip through memory cost more than the uneven finish of whole streams: 32 sequences x 8 KV heads of 512 to
+// 2048 tokens measured 31 us against 36).  Only bounds known on the host decide: max_partitions * partition_size
+// bounds every context.
+static bool step_prefers_single_pass(int B, int Hkv, int partition_size, int max_partitions) {
+    const long long streams = (long long)B * Hkv, bound = (long long)max_partitions * partition_size;
+    const int sms = sm_count();
+    return sms > 0 && bound <= 2048 && 2 * streams >= 3ll * sms && streams <= 4ll * sms;
+}
 
 int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void* v_new,
                         const int64_t* slot_mapping, void* k_cache, void* v_cache, const int32_t* block_tables,
                         int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes,
                         float scale, int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks,
-                        int partition_size, void* workspace, int max_partitions, int dtype, void* stream) {
+                        int partition_size, void* workspace, size_t workspace_bytes, int max_partitions, int dtype,
+                        void* stream) {
     if (!out) return B == 0 ? OPT_GQA_OK : OPT_GQA_ERR_NULL;
     if (partition_size > 0 && !workspace && B > 0) return OPT_GQA_ERR_NULL;
+    if (dtype_ok(dtype) && shape_ok(Hq, Hkv, D, bs) &&
+        workspace_bytes < step_workspace_need(B, Hq, Hkv, D, partition_size, max_partitions, dtype))
+        return OPT_GQA_ERR_SHAPE;
     int rc;
+    if (dtype == OPT_GQA_BF16 && partition_size > 0 && B > 0 && shape_ok(Hq, Hkv, D, bs) && max_partitions > 0 &&
+        step_prefers_single_pass(B, Hkv, partition_size, max_partitions)) {
+        if (num_blocks <= 0 || max_blocks_per_seq <= 0 || B > 65535 || partition_size % 16 != 0) return OPT_GQA_ERR_SHAPE;
+        if (!q || !k_new || !v_new || !k_cache || !v_cache || !slot_mapping || !block_tables || !context_lens)
+            return OPT_GQA_ERR_NULL;
+        if (!aligned16(out) || !aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) ||
+            !aligned16(v_cache))
+            return OPT_GQA_ERR_ALIGN;
+        int* status = device_status_ptr();
+        if (!status) return OPT_GQA_ERR_CUDA;
+        const FusedAppend fa = {k_new, v_new, k_cache, v_cache, slot_mapping};
+        return launch_decode_tc(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
+                                scale, B, Hq, Hkv, D, bs, num_blocks, 0, nullptr, nullptr, 1, status,
+                                static_cast<cudaStream_t>(stream), &fa);
+    }
     if (dtype == OPT_GQA_BF16 && partition_size > 0 && B > 0) {
         // bf16 split.  With few (sequence, KV head) streams the streaming kernel stores the new tokens itself, each
         // just before the tile that holds it is fetched, and the separate launch is saved; with thousands of
@@ -287,6 +333,8 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
             if (!k_new || !v_new || !k_cache || !v_cache || !slot_mapping) return OPT_GQA_ERR_NULL;
             if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache))
                 return OPT_GQA_ERR_ALIGN;
+            // nothing may be enqueued if the merge's own checks would fail afterwards
+            if (!aligned16(out)) return OPT_GQA_ERR_ALIGN;
         } else {
             rc = opt_gqa_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, B, Hkv, D, bs, num_blocks, dtype,
                                       stream);
@@ -294,18 +342,18 @@ int opt_gqa_decode_step(void* out, const void* q, const void* k_new, const void*
         }
         const FusedAppend fa = {k_new, v_new, k_cache, v_cache, slot_mapping};
         rc = decode_balanced_checked(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
-                                     scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, max_partitions, 0,
-                                     dtype, stream, fuse ? &fa : nullptr);
+                                     scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, workspace_bytes,
+                                     max_partitions, 0, dtype, stream, fuse ? &fa : nullptr);
         if (rc != OPT_GQA_OK) return rc;
-        return opt_gqa_paged_attention_reduce_balanced(out, workspace, context_lens, B, Hq, Hkv, D, partition_size,
-                                                       max_partitions, dtype, stream);
+        return opt_gqa_paged_attention_reduce_balanced(out, workspace, workspace_bytes, context_lens, B, Hq, Hkv, D,
+                                                       partition_size, max_partitions, dtype, stream);
     }
+    // one partial per partition: partial_out [B, Hq, max_partitions, D] followed by partial_lse
+    const size_t part_rows = (size_t)(B > 0 ? B : 0) * (size_t)(Hq > 0 ? Hq : 0) * (size_t)(max_partitions > 0 ? max_partitions : 0);
     rc = opt_gqa_cache_append(k_new, v_new, k_cache, v_cache, slot_mapping, B, Hkv, D, bs, num_blocks, dtype, stream);
     if (rc != OPT_GQA_OK) return rc;
     float* partial_out = static_cast<float*>(workspace);
-    float* partial_lse =
-        partial_out ? partial_out + (size_t)(B > 0 ? B : 0) * Hq * (max_partitions > 0 ? max_partitions : 0) * D
-                    : nullptr;
+    float* partial_lse = partial_out ? partial_out + part_rows * (size_t)(D > 0 ? D : 0) : nullptr;
     rc = opt_gqa_paged_attention_decode(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                                         alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size,
                                         partial_out, partial_lse, max_partitions, dtype, stream);
@@ -395,7 +443,7 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
                              const int32_t* context_lens_host, void* staging, void* k_cache, void* v_cache,
                              int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
                              int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
-                             int max_partitions, int dtype, void* stream) {
+                             size_t workspace_bytes, int max_partitions, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0) return OPT_GQA_ERR_SHAPE;
     if (B == 0) return OPT_GQA_OK;
@@ -403,6 +451,12 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
         !context_lens_host || !staging)
         return OPT_GQA_ERR_NULL;
     if ((reinterpret_cast<uintptr_t>(staging) & 255u) != 0) return OPT_GQA_ERR_ALIGN;
+    // what the step itself would refuse is refused here, before the transfers are enqueued
+    if (partition_size < 0 || partition_size % 16 != 0 || (partition_size > 0 && max_partitions <= 0) || num_blocks <= 0)
+        return OPT_GQA_ERR_SHAPE;
+    if (partition_size > 0 && !workspace) return OPT_GQA_ERR_NULL;
+    if (!k_cache || !v_cache) return OPT_GQA_ERR_NULL;
+    if (workspace_bytes < step_workspace_need(B, Hq, Hkv, D, partition_size, max_partitions, dtype)) return OPT_GQA_ERR_SHAPE;
     StagingLayout L;
     if (!staging_layout(B, Hq, Hkv, D, max_blocks_per_seq, dtype, &L)) return OPT_GQA_ERR_SHAPE;
     const size_t es = dtype == OPT_GQA_FP32 ? 4 : 2;
@@ -449,7 +503,8 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
                                  reinterpret_cast<const int64_t*>(st + L.slots), k_cache, v_cache,
                                  reinterpret_cast<const int32_t*>(st + L.tables), max_blocks_per_seq,
                                  reinterpret_cast<const int32_t*>(st + L.lens), alibi_slopes, scale, B, Hq, Hkv, D,
-                                 bs, num_blocks, partition_size, workspace, max_partitions, dtype, stream);
+                                 bs, num_blocks, partition_size, workspace, workspace_bytes, max_partitions, dtype,
+                                 stream);
     if (rc != OPT_GQA_OK) return rc;
     if (!pinned && cudaMemcpyAsync(out_host, st + L.out, qb, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
         return OPT_GQA_ERR_CUDA;

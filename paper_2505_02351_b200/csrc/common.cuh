@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "opt_gqa.h"
 
 namespace optgqa {
@@ -67,12 +69,13 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t par
     return done != 0;
 }
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     do {
         if (mbar_try_wait_parked(bar, parity, 4000)) return true;
-    } while (clock64() - start < kWaitLimitCycles);
+    } while (clock64() - start < limit_cycles);
     atomicExch(status, OPT_GQA_ERR_TIMEOUT);
     return false;
 }
@@ -163,6 +166,27 @@ struct Store<__nv_bfloat16> {
 // Address of the current device's status word (api.cu); nullptr if the runtime refuses.
 int* device_status_ptr();
 
+// Multiprocessors of the current device (cached per device); 0 if the runtime refuses (decode_stream.cu).
+int sm_count();
+
+// Per-device host-side caches (symbol addresses, attribute flags, SM counts) are arrays of atomics indexed by the
+// device ordinal: two host threads making their first call together both do the (idempotent) set-up and store the
+// same value, without a data race.
+constexpr int kMaxDevices = 64;
+
+// Raises the dynamic shared memory limit of `kernel` once per device.  `done` is the launcher's own
+// `static std::atomic<bool> [kMaxDevices]`.
+template <typename Kernel>
+inline bool ensure_smem_limit(Kernel kernel, int bytes, std::atomic<bool>* done) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached && done[dev].load(std::memory_order_acquire)) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (cached) done[dev].store(true, std::memory_order_release);
+    return true;
+}
+
 // ----------------------------------------------------------------------------- host-side launchers (one per .cu)
 int launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                         const int64_t* slot_mapping, int T, int Hkv, int D, int bs, int dtype,
@@ -170,15 +194,8 @@ int launch_cache_append(const void* k_new, const void* v_new, void* k_cache, voi
 
 int launch_decode(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                   int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
-                  int B, int Hq, int Hkv, int D, int bs, int partition_size, float* partial_out,
+                  int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size, float* partial_out,
                   float* partial_lse, int max_partitions, int dtype, int* device_status, cudaStream_t stream);
-
-// bf16 only: the query group as rows of tensor-core tiles (decode_tc.cu).
-int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
-                     int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
-                     int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                     float* partial_out, float* partial_lse, int max_partitions, int* device_status,
-                     cudaStream_t stream);
 
 // Workspace of the balanced split (bf16 caches, partition_size > 0).  The stream of 16-token tiles
 // (sequence, KV head, partition order) is cut into one range per worker at TILE granularity; a piece is the
@@ -214,14 +231,20 @@ struct FusedAppend {
     const int64_t* slot_mapping;    // [B]; negative: nothing to store
 };
 
+// bf16 only: the query group as rows of tensor-core tiles (decode_tc.cu).  append != nullptr: see FusedAppend.
+int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
+                     int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
+                     int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
+                     float* partial_out, float* partial_lse, int max_partitions, int* device_status,
+                     cudaStream_t stream, const FusedAppend* append = nullptr);
+
 // bf16, partition_size > 0, balanced split into `workspace`: persistent streaming kernel, one worker per warp
-// (decode_stream.cu).  partial_out / partial_lse are unused (one partial per partition is launch_decode_tc's job).
-// append != nullptr (balanced split only): see FusedAppend.
+// (decode_stream.cu).  append != nullptr: see FusedAppend.
 int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                          int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                         float* partial_out, float* partial_lse, void* workspace, int max_partitions, int window,
-                         int* device_status, cudaStream_t stream, const FusedAppend* append = nullptr);
+                         void* workspace, int max_partitions, int window, int* device_status, cudaStream_t stream,
+                         const FusedAppend* append = nullptr);
 
 // Workers (warps) of the grid that launch_decode_stream uses for the balanced split of these sizes on the current
 // device; 0 if the device cannot be queried.

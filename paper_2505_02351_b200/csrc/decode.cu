@@ -32,6 +32,7 @@ struct DecodeParams {
     int* status;
     float scale;
     int max_blocks;
+    int num_blocks;
     int Hq;
     int Hkv;
     int bs;
@@ -148,7 +149,10 @@ decode_kernel(const DecodeParams p) {
     const int t1 = split ? min(t0 + p.partition_size, n) : n;
 
     if (t0 >= t1) {
-        // Empty range.  A single-pass call still owes zero rows for an empty sequence.
+        // Empty range.  A single-pass call still owes zero rows for an empty sequence.  The wait comes first all the
+        // same: an earlier kernel of the stream may still be reading out, and a grid none of whose CTAs waited could
+        // finish before its predecessor.
+        grid_dependency_wait();
         if (!split) {
             T* o = static_cast<T*>(p.out) + ((size_t)s * p.Hq + (size_t)kvh * G) * D;
             for (int e = threadIdx.x; e < G * D; e += blockDim.x) store_out(o + e, 0.f);
@@ -180,7 +184,10 @@ decode_kernel(const DecodeParams p) {
     // Physical pages of this warp's tiles, 32 at a time, one block ahead of the issue index.
     auto load_pages = [&](int kb) -> int {
         int k = kb + lane;
-        return k < cnt ? __ldg(table + (first_tile + warp + k * kWarps) / tpp) : 0;
+        // Index held inside the table and page id inside the pool: index data that breaks the caller's promises
+        // gives a wrong row, not a copy from outside the cache.
+        const int page = k < cnt ? __ldg(table + min((first_tile + warp + k * kWarps) / tpp, p.max_blocks - 1)) : 0;
+        return min(max(page, 0), p.num_blocks - 1);
     };
     int pages_cur = load_pages(0), pages_next = load_pages(32), blk = 0;
 
@@ -374,15 +381,8 @@ decode_kernel(const DecodeParams p) {
 template <typename T, int D, int G>
 static int launch_one(const DecodeParams& p, int B, cudaStream_t stream) {
     using C = DecodeCfg<T, D, G>;
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
-    if (dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(decode_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) !=
-            cudaSuccess)
-            return OPT_GQA_ERR_CUDA;
-        configured[dev] = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];
+    if (!ensure_smem_limit(decode_kernel<T, D, G>, C::SMEM, configured)) return OPT_GQA_ERR_CUDA;
     dim3 grid(p.partition_size > 0 ? p.max_partitions : 1, p.Hkv, B);
     return launch_dependent(decode_kernel<T, D, G>, grid, dim3(kWarps * 32), C::SMEM, stream, p);
 }
@@ -400,9 +400,11 @@ static int launch_g(const DecodeParams& p, int B, int G, cudaStream_t stream) {
 
 int launch_decode(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                   int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
-                  int B, int Hq, int Hkv, int D, int bs, int partition_size, float* partial_out,
+                  int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size, float* partial_out,
                   float* partial_lse, int max_partitions, int dtype, int* device_status, cudaStream_t stream) {
+    if (num_blocks <= 0 || num_blocks > 0x7fffffffll) return OPT_GQA_ERR_SHAPE;
     DecodeParams p;
+    p.num_blocks = (int)num_blocks;
     p.out = out;
     p.q = q;
     p.k_cache = static_cast<const char*>(k_cache);

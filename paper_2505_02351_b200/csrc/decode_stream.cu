@@ -2,17 +2,16 @@
 // streaming form (Algorithm 2, "Compute context attention with caches"; Eq. 3-5; the
 // long-sequence partitioning described before Eq. 1).
 //
-// Work items are (sequence, KV head, context partition) triples, each producing one
-// normalised partial result and its log-sum-exp for all G query heads of the group
-// ("Shared Key-Value": a K/V tile is brought on-chip once for the whole group).  The
-// grid is persistent: every warp is an independent worker with a private ring of
-// 16-token K/V tiles fetched by 2-D TMA (128-byte swizzle).  The items, laid end to
-// end in (sequence, KV head, partition) order and measured in tiles, are cut into one
-// contiguous range per worker; a worker owns the items that start inside its range and
-// streams them back to back, so the ring never drains between items: page ids, the
-// query rows and the slopes of the next item are fetched while the current one is
-// still being consumed.  The cut is computed by every warp from context_lens alone
-// (two coalesced passes), so there is no scheduler state in global memory.
+// The streams (sequence, KV head), each ceil(n / 16) tiles of 16 tokens long, are laid end to end and cut
+// into one contiguous range per worker at tile granularity, so that every SM streams the same number of
+// cache bytes whatever the mix of lengths.  A piece is the part of one context partition that lies inside
+// one range; it produces a normalised partial result and its log-sum-exp for all G query heads of the
+// group ("Shared Key-Value": a K/V tile is brought on-chip once for the whole group), and the merge
+// (reduce.cu) combines the pieces of a stream.  The grid is persistent: every warp is an independent worker
+// with a private ring of K/V tiles fetched by 2-D TMA (128-byte swizzle) and streams its pieces back to
+// back, so the ring never drains between pieces: page ids, the query rows and the slopes of the next piece
+// are fetched while the current one is still being consumed.  The cut is computed by every warp from
+// context_lens alone (two coalesced passes), so there is no scheduler state in global memory.
 //
 // When the caller hands over the step's new K/V rows (Algorithm 2, "Store reshaped K, V into C_K, C_V"), the
 // worker that is about to fetch the tile holding a sequence's last position stores that sequence's new token
@@ -34,19 +33,10 @@ namespace optgqa {
 
 namespace {
 
-#ifndef OPT_GQA_STREAM_WARPS
-#define OPT_GQA_STREAM_WARPS 4
-#endif
-#ifndef OPT_GQA_STREAM_STAGES
-#define OPT_GQA_STREAM_STAGES 2
-#endif
-#ifndef OPT_GQA_STREAM_CTAS
-#define OPT_GQA_STREAM_CTAS 2
-#endif
 constexpr int kTileTok = 16;                     // tokens per tile (one ring stage holds a K tile and a V tile)
-constexpr int kWarps = OPT_GQA_STREAM_WARPS;     // workers per CTA
-constexpr int kStages = OPT_GQA_STREAM_STAGES;   // ring depth per worker
-constexpr int kCtasPerSm = OPT_GQA_STREAM_CTAS;
+constexpr int kWarps = 4;                        // workers per CTA
+constexpr int kStages = 2;                       // ring depth per worker
+constexpr int kCtasPerSm = 2;
 constexpr int kDescSlots = 4;                    // item descriptors a worker keeps (>= items between prefetch and use)
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kMaxSlack = 8.f;                // log2 units by which a score may exceed the running reference maximum
@@ -56,10 +46,10 @@ struct StreamParams {
     const int32_t* block_tables;
     const int32_t* context_lens;
     const float* slopes;
-    float* partial_out;
+    float* partial_out;     // rows of the pieces (see balanced_layout)
     float* partial_lse;
-    long long* header;      // balanced split: {tiles in the stream, workers}
-    long long* seq_info;    // balanced split: per sequence {tiles, partitions} of one head over the earlier sequences
+    long long* header;      // {tiles in the stream, workers}
+    long long* seq_info;    // per sequence {tiles, partitions} of one head over the earlier sequences
     int* status;
     float scale;
     int B;
@@ -69,7 +59,7 @@ struct StreamParams {
     int bs;
     int partition_size;
     int max_partitions;
-    int window;             // > 0: only the last `window` keys of each sequence are attended to (balanced split only)
+    int window;             // > 0: only the last `window` keys of each sequence are attended to
     // fused store of the step's new tokens (all null when the cache already holds them)
     const uint4* k_new;
     const uint4* v_new;
@@ -125,7 +115,7 @@ struct StreamCursor {
     long long parts_before; // sum of `parts` over earlier sequences (one head)
 };
 
-template <int D, int G, bool kBalanced>
+template <int D, int G>
 __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
 decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                      const StreamParams p) {
@@ -145,7 +135,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     // partitions are counted from there.
     auto first_tile_of = [&](int n) { return p.window > 0 ? max(0, n - p.window) / kTileTok : 0; };
     auto tiles_of = [&](int n) { return (n + kTileTok - 1) / kTileTok - first_tile_of(n); };
-    const int* __restrict__ lens = p.context_lens;         // an input of the step: not written by the preceding grid
+    const int* __restrict__ lens = p.context_lens;         // read before the dependency wait: see the ordering contract
+    // Entry of a sequence's page table that holds token `tok`.  Held below max_blocks, so that a context length that
+    // breaks the caller's promise (n_s <= max_blocks * bs) gives a wrong row and not an access outside the table.
+    auto table_index = [&](int tok) { return min(tok / p.bs, p.max_blocks - 1); };   // max_blocks >= 1 (host check)
     if (lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
@@ -164,7 +157,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     // Never more workers than tiles, so that every worker's range holds at least one tile.
     const long long grid_workers = (long long)gridDim.x * kWarps, me = (long long)blockIdx.x * kWarps + warp;
     const long long workers = total < grid_workers ? (total > 0 ? total : 1) : grid_workers;
-    if (kBalanced && me == 0) {
+    if (me == 0) {
         grid_dependency_wait();     // the previous reader of the workspace must be done
         if (lane == 0) {
             p.header[0] = total;
@@ -225,13 +218,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             cur.parts = (cur.tiles + P16 - 1) / P16;
         }
     };
-    if (!kBalanced && cur.jt % P16 != 0) {
-        // whole partitions only: the first one that starts at or after lo
-        const int adv = min(P16 - cur.jt % P16, cur.tiles - cur.jt);
-        cur.jt += adv;
-        cur.pos += adv;
-        if (cur.jt == cur.tiles) next_stream();
-    }
     auto cur_valid = [&]() { return cur.s < p.B && cur.pos < hi; };
     if (!cur_valid()) return;
 
@@ -246,30 +232,23 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     __syncwarp();
 
     // Describes the piece under `cur` in slot (piece & 3), starts the loads of its first 32 page ids, moves `cur`
-    // on.  A piece is the part of one partition that lies inside this worker's range (kBalanced) or one whole
-    // partition (otherwise).  desc[2i] = {s, kvh, n, first tile in the stream}, desc[2i+1] = {tiles, row of the
+    // on.  A piece is the part of one partition that lies inside this worker's range.  desc[2i] = {s, kvh, n, first tile in the stream}, desc[2i+1] = {tiles, row of the
     // partial result of the group's first head}; tiles are numbered from the sequence's token 0.
     int pieces = 0;               // pieces described so far
     int pages_nxt = 0;            // lane l: physical page of tile l of the piece described last
     auto describe_next = [&]() {
         const int part = cur.jt / P16;
-        int len = min((part + 1) * P16, cur.tiles) - cur.jt;
-        int obase;
-        if (kBalanced) {
-            len = (int)min((long long)len, hi - cur.pos);
-            // pieces are numbered by (partition index in the end-to-end order) + (worker index): both only grow
-            obase = (int)((cur.parts_before * p.Hkv + (long long)cur.kvh * cur.parts + part + me) * G);
-            if (lane == 0 && cur.kvh == 0 && cur.jt == 0) {
-                p.seq_info[2 * cur.s] = cur.tiles_before;
-                p.seq_info[2 * cur.s + 1] = cur.parts_before;
-            }
-            // Where this range and a partition end together inside a stream, the next piece is two numbers on:
-            // mark the number in between as empty, so that the merge can sweep the stream's numbers without gaps.
-            if (cur.pos + len == hi && cur.jt + len < cur.tiles && (cur.jt + len) % P16 == 0 && lane < G)
-                p.partial_lse[obase + G + lane] = -INFINITY;
-        } else {
-            obase = (cur.s * p.Hq + cur.kvh * G) * p.max_partitions + part;
+        const int len = (int)min((long long)(min((part + 1) * P16, cur.tiles) - cur.jt), hi - cur.pos);
+        // pieces are numbered by (partition index in the end-to-end order) + (worker index): both only grow
+        const int obase = (int)((cur.parts_before * p.Hkv + (long long)cur.kvh * cur.parts + part + me) * G);
+        if (lane == 0 && cur.kvh == 0 && cur.jt == 0) {
+            p.seq_info[2 * cur.s] = cur.tiles_before;
+            p.seq_info[2 * cur.s + 1] = cur.parts_before;
         }
+        // Where this range and a partition end together inside a stream, the next piece is two numbers on:
+        // mark the number in between as empty, so that the merge can sweep the stream's numbers without gaps.
+        if (cur.pos + len == hi && cur.jt + len < cur.tiles && (cur.jt + len) % P16 == 0 && lane < G)
+            p.partial_lse[obase + G + lane] = -INFINITY;
         if (lane == 0) {
             desc[2 * (pieces & (kDescSlots - 1))] = make_int4(cur.s, cur.kvh, cur.n, first_tile_of(cur.n) + cur.jt);
             desc[2 * (pieces & (kDescSlots - 1)) + 1] = make_int4(len, obase, 0, 0);
@@ -277,7 +256,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         // the piece is streamed from its last tile backwards: page ids of its last block of 32 tiles first
         const int blk = (len - 1) & ~31;
         const int tok = (first_tile_of(cur.n) + cur.jt + blk + lane) * kTileTok;
-        pages_nxt = blk + lane < len ? __ldg(p.block_tables + (size_t)cur.s * p.max_blocks + tok / p.bs) : 0;
+        pages_nxt = blk + lane < len ? __ldg(p.block_tables + (size_t)cur.s * p.max_blocks + table_index(tok)) : 0;
         ++pieces;
         cur.pos += len;
         cur.jt += len;
@@ -307,12 +286,15 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             is_kvh = d0.y;
             is_tile0 = d0.w;
             is_last_tile = (d0.z - 1) / kTileTok;          // the tile that holds the sequence's newest token
+            // q may be the output of the kernel that precedes this one in the stream (the Q/K/V projection, which
+            // lets its dependents start early): it is read only after the dependency wait, and from L2, never through
+            // a non-coherent path that could hold a line fetched before that kernel's stores.
             const uint32_t* qh = reinterpret_cast<const uint32_t*>(
                 p.q + ((size_t)d0.x * p.Hq + (size_t)d0.y * G + (g < G ? g : 0)) * D);
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
-                q_nxt[ks][0] = g < G ? __ldg(qh + ks * 8 + t) : 0u;
-                q_nxt[ks][1] = g < G ? __ldg(qh + ks * 8 + 4 + t) : 0u;
+                q_nxt[ks][0] = g < G ? __ldcg(qh + ks * 8 + t) : 0u;
+                q_nxt[ks][1] = g < G ? __ldcg(qh + ks * 8 + 4 + t) : 0u;
             }
 #pragma unroll
             for (int c = 0; c < 2; ++c)
@@ -321,7 +303,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         } else if (((is_ntile - 1 - is_j) & 31) == 31) {
             // pieces longer than 512 tokens: the page ids of the block of 32 tiles below
             const int tok = (is_tile0 + (is_ntile - 32 - is_j) + lane) * kTileTok;
-            pages_cur = __ldg(p.block_tables + (size_t)is_s * p.max_blocks + tok / p.bs);
+            pages_cur = __ldg(p.block_tables + (size_t)is_s * p.max_blocks + table_index(tok));
         }
         const int is_r = is_ntile - 1 - is_j;      // tile inside the piece: from the last one backwards
         if (p.k_new && is_tile0 + is_r == is_last_tile) {
@@ -367,17 +349,17 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     };
 
     {
-        // While the preceding grid drains: bring what the first piece needs and that grid does not write (page ids,
-        // query rows) towards this SM, so that the first copies can be issued right after the wait.
+        // While the preceding grid drains: bring the first piece's page ids towards this SM (the page table is
+        // complete before the call, see the ordering contract in the header), and ask L2 -- the point of coherence,
+        // where a line can never be stale -- for the query rows, which the preceding grid may still be writing.
         const int part = cur.jt / P16;
-        int len = min((part + 1) * P16, cur.tiles) - cur.jt;
-        if (kBalanced) len = (int)min((long long)len, hi - cur.pos);
+        const int len = (int)min((long long)(min((part + 1) * P16, cur.tiles) - cur.jt), hi - cur.pos);
         const int blk = (len - 1) & ~31;
         const int tok = (first_tile_of(cur.n) + cur.jt + blk + lane) * kTileTok;
         if (blk + lane < len)
-            asm volatile("prefetch.global.L1 [%0];" ::"l"(p.block_tables + (size_t)cur.s * p.max_blocks + tok / p.bs));
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(p.block_tables + (size_t)cur.s * p.max_blocks + table_index(tok)));
         if (lane < G * D * 2 / 128)
-            asm volatile("prefetch.global.L1 [%0];" ::"l"(
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(
                 reinterpret_cast<const char*>(p.q + ((size_t)cur.s * p.Hq + (size_t)cur.kvh * G) * D) + lane * 128));
     }
     grid_dependency_wait();     // the cache may still be receiving this step's appended tokens
@@ -390,7 +372,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     float o[MT][4];
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     int cs_j = 0, cs_ntile = 0, cs_n = 0, cs_tile0 = 0, cs_obase = 0;
-    const int ostride = kBalanced ? 1 : p.max_partitions;     // distance between the rows of consecutive heads
     const int lrow = lane & 7, lmat = lane >> 3;
     bool ok = true;
 
@@ -512,7 +493,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             const float L0 = group_sum(l0), L1 = group_sum(l1);
             const float i0 = 1.f / L0, i1 = 1.f / L1;
             if (2 * t < G) {
-                const size_t row = (size_t)cs_obase + (size_t)(2 * t) * ostride;
+                const size_t row = (size_t)cs_obase + (size_t)(2 * t);
                 float* po = p.partial_out + row * D;
 #pragma unroll
                 for (int i = 0; i < MT; ++i) {
@@ -522,7 +503,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 if (g == 0) st_global_hint(p.partial_lse + row, (m0 + lg2(L0)) * kLn2, keep);
             }
             if (2 * t + 1 < G) {
-                const size_t row = (size_t)cs_obase + (size_t)(2 * t + 1) * ostride;
+                const size_t row = (size_t)cs_obase + (size_t)(2 * t + 1);
                 float* po = p.partial_out + row * D;
 #pragma unroll
                 for (int i = 0; i < MT; ++i) {
@@ -548,94 +529,84 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     }
 }
 
-int sm_count() {
-    static int counts[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
-    if (!counts[dev] && cudaDeviceGetAttribute(&counts[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    return counts[dev];
-}
-
-// One resident wave; never more workers than there could be units of work (whole partitions, or 16-token tiles in the
-// balanced split, whose ranges are cut at tile granularity), nor than the workspace has room for.  In the balanced
-// split a grid that leaves some SMs with one CTA and others with two would undo the balance.
-long long stream_grid_ctas(int B, int Hkv, int max_partitions, int partition_size, bool balanced) {
+// One resident wave; never more workers than there could be 16-token tiles (the ranges are cut at tile granularity),
+// nor than the workspace has room for.  A grid that leaves some SMs with one CTA and others with two would undo the
+// balance.
+long long stream_grid_ctas(int B, int Hkv, int max_partitions, int partition_size) {
     const int sms = sm_count();
     if (sms <= 0) return 0;
-    long long items = (long long)B * Hkv * max_partitions;
-    if (balanced) items *= partition_size / kTileTok;
+    const long long items = (long long)B * Hkv * max_partitions * (partition_size / kTileTok);
     long long ctas = (items + kWarps - 1) / kWarps;
     if (ctas > (long long)sms * kCtasPerSm) ctas = (long long)sms * kCtasPerSm;
     if (ctas > kBalancedMaxWorkers / kWarps) ctas = kBalancedMaxWorkers / kWarps;
     return ctas;
 }
 
-template <int D, int G, bool kBalanced>
+template <int D, int G>
 int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams& p, cudaStream_t stream) {
     using C = StreamCfg<D>;
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
-    if (dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(decode_stream_kernel<D, G, kBalanced>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 C::SMEM) != cudaSuccess)
-            return OPT_GQA_ERR_CUDA;
-        configured[dev] = true;
-    }
-    const long long ctas = stream_grid_ctas(p.B, p.Hkv, p.max_partitions, p.partition_size, kBalanced);
+    static std::atomic<bool> configured[kMaxDevices];
+    if (!ensure_smem_limit(decode_stream_kernel<D, G>, C::SMEM, configured)) return OPT_GQA_ERR_CUDA;
+    const long long ctas = stream_grid_ctas(p.B, p.Hkv, p.max_partitions, p.partition_size);
     if (ctas <= 0) return OPT_GQA_ERR_CUDA;
-    return launch_dependent(decode_stream_kernel<D, G, kBalanced>, dim3((unsigned)ctas), dim3(kWarps * 32), C::SMEM,
-                            stream, mk, mv, p);
+    return launch_dependent(decode_stream_kernel<D, G>, dim3((unsigned)ctas), dim3(kWarps * 32), C::SMEM, stream, mk,
+                            mv, p);
 }
 
-template <int D, bool kBalanced>
+template <int D>
 int launch_g(const CUtensorMap& mk, const CUtensorMap& mv, const StreamParams& p, int G, cudaStream_t stream) {
     switch (G) {
-        case 1: return launch_one<D, 1, kBalanced>(mk, mv, p, stream);
-        case 2: return launch_one<D, 2, kBalanced>(mk, mv, p, stream);
-        case 4: return launch_one<D, 4, kBalanced>(mk, mv, p, stream);
-        case 8: return launch_one<D, 8, kBalanced>(mk, mv, p, stream);
+        case 1: return launch_one<D, 1>(mk, mv, p, stream);
+        case 2: return launch_one<D, 2>(mk, mv, p, stream);
+        case 4: return launch_one<D, 4>(mk, mv, p, stream);
+        case 8: return launch_one<D, 8>(mk, mv, p, stream);
     }
     return OPT_GQA_ERR_SHAPE;
 }
 
 }  // namespace
 
-long long stream_grid_workers(int B, int Hkv, int max_partitions, int partition_size) {
-    return stream_grid_ctas(B, Hkv, max_partitions, partition_size, true) * kWarps;
+int sm_count() {
+    static std::atomic<int> counts[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    int c = counts[dev].load(std::memory_order_relaxed);
+    if (!c) {
+        if (cudaDeviceGetAttribute(&c, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        counts[dev].store(c, std::memory_order_relaxed);
+    }
+    return c;
 }
 
-// The balanced split: pieces and bookkeeping go to `workspace` (see balanced_layout).  (The kernel can also own whole
-// partitions and write one partial result per partition to partial_out / partial_lse -- kBalanced = false -- but
-// whole partitions are balanced better by one CTA per partition, decode_tc.cu, which is what the library launches.)
+long long stream_grid_workers(int B, int Hkv, int max_partitions, int partition_size) {
+    return stream_grid_ctas(B, Hkv, max_partitions, partition_size) * kWarps;
+}
+
+// Pieces and bookkeeping go to `workspace` (see balanced_layout).  One partial per whole partition is the tile
+// kernel's job (decode_tc.cu, one CTA per partition).
 int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                          int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                          int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
-                         float* partial_out, float* partial_lse, void* workspace, int max_partitions, int window,
-                         int* device_status, cudaStream_t stream, const FusedAppend* append) {
+                         void* workspace, int max_partitions, int window, int* device_status, cudaStream_t stream,
+                         const FusedAppend* append) {
+    if (!workspace) return OPT_GQA_ERR_NULL;
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
     CUtensorMap mk, mv;
     if (!make_cache_map(&mk, k_cache, rows, D, kTileTok) || !make_cache_map(&mv, v_cache, rows, D, kTileTok))
         return OPT_GQA_ERR_CUDA;
+    const BalancedLayout L = balanced_layout(B, Hq, Hkv, D, max_partitions);
+    if (L.rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
+    char* ws = static_cast<char*>(workspace);
     StreamParams p;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.block_tables = block_tables;
     p.context_lens = context_lens;
     p.slopes = alibi_slopes;
-    p.partial_out = partial_out;
-    p.partial_lse = partial_lse;
-    p.header = nullptr;
-    p.seq_info = nullptr;
-    if (workspace) {
-        const BalancedLayout L = balanced_layout(B, Hq, Hkv, D, max_partitions);
-        if (L.rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
-        char* ws = static_cast<char*>(workspace);
-        p.header = reinterpret_cast<long long*>(ws + L.header);
-        p.seq_info = reinterpret_cast<long long*>(ws + L.seq_info);
-        p.partial_lse = reinterpret_cast<float*>(ws + L.lse);
-        p.partial_out = reinterpret_cast<float*>(ws + L.out);
-    }
+    p.header = reinterpret_cast<long long*>(ws + L.header);
+    p.seq_info = reinterpret_cast<long long*>(ws + L.seq_info);
+    p.partial_lse = reinterpret_cast<float*>(ws + L.lse);
+    p.partial_out = reinterpret_cast<float*>(ws + L.out);
     p.status = device_status;
     p.scale = scale;
     p.B = B;
@@ -645,17 +616,15 @@ int launch_decode_stream(const void* q, const void* k_cache, const void* v_cache
     p.bs = bs;
     p.partition_size = partition_size;
     p.max_partitions = max_partitions;
-    p.window = workspace ? window : 0;
-    const bool fuse = workspace && append;
-    p.k_new = fuse ? static_cast<const uint4*>(append->k_new) : nullptr;
-    p.v_new = fuse ? static_cast<const uint4*>(append->v_new) : nullptr;
-    p.k_cache_w = fuse ? static_cast<uint4*>(append->k_cache) : nullptr;
-    p.v_cache_w = fuse ? static_cast<uint4*>(append->v_cache) : nullptr;
-    p.slot_mapping = fuse ? append->slot_mapping : nullptr;
+    p.window = window;
+    p.k_new = append ? static_cast<const uint4*>(append->k_new) : nullptr;
+    p.v_new = append ? static_cast<const uint4*>(append->v_new) : nullptr;
+    p.k_cache_w = append ? static_cast<uint4*>(append->k_cache) : nullptr;
+    p.v_cache_w = append ? static_cast<uint4*>(append->v_cache) : nullptr;
+    p.slot_mapping = append ? append->slot_mapping : nullptr;
     const int G = Hq / Hkv;
-    if (!workspace) return OPT_GQA_ERR_NULL;    // one partial per partition: decode_tc.cu (one CTA per partition)
-    if (D == 128) return launch_g<128, true>(mk, mv, p, G, stream);
-    if (D == 64) return launch_g<64, true>(mk, mv, p, G, stream);
+    if (D == 128) return launch_g<128>(mk, mv, p, G, stream);
+    if (D == 64) return launch_g<64>(mk, mv, p, G, stream);
     return OPT_GQA_ERR_SHAPE;
 }
 

@@ -21,9 +21,6 @@ namespace optgqa {
 
 namespace {
 
-#ifndef OPT_GQA_TC_STAGES
-#define OPT_GQA_TC_STAGES 2
-#endif
 // Warps per CTA (each with a private ring) and CTAs per SM the register budget is held to, for the two uses of the
 // kernel.  One CTA per (sequence, KV head) has the whole context to itself: eight warps, one CTA per SM.  One CTA per
 // (sequence, KV head, partition) has a few hundred tokens: two warps, six CTAs per SM, so that the CTA scheduler has
@@ -32,7 +29,7 @@ namespace {
 constexpr int kWarpsSingle = 8, kCtasSingle = 1;
 constexpr int kWarpsSplit = 2, kCtasSplit = 6;
 constexpr int kTileTok = 16;                 // tokens per tile (one ring stage holds a K tile and a V tile)
-constexpr int kStages = OPT_GQA_TC_STAGES;   // ring depth per warp
+constexpr int kStages = 2;                   // ring depth per warp
 constexpr unsigned kFull = 0xffffffffu;
 
 struct TcParams {
@@ -51,6 +48,13 @@ struct TcParams {
     int bs;
     int partition_size;
     int max_partitions;
+    int B;
+    // fused store of the step's new tokens (all null when the cache already holds them)
+    const uint4* k_new;
+    const uint4* v_new;
+    uint4* k_cache_w;
+    uint4* v_cache_w;
+    const int64_t* slot_mapping;
 };
 
 template <int D, int G, int kWarps>
@@ -93,15 +97,30 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
     const uint64_t read_once = l2_policy_evict_first();     // every K/V byte is read exactly once
     const uint64_t keep = l2_policy_evict_last();           // the partial results are read by the merge that follows
-    const int part = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+    // Work item of this CTA.  The sequence index runs fastest and the partition index slowest, so that the grid ends
+    // with the high partition numbers, which only the longest sequences have: the last CTAs to start are few and short.
+    const int s = blockIdx.x % p.B, kvh = (blockIdx.x / p.B) % p.Hkv, part = blockIdx.x / (p.B * p.Hkv);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;      // fragment row (query head of the group) and column pair
-    const int n = p.context_lens[s];
     const bool split = p.partition_size > 0;
     const int t0 = split ? part * p.partition_size : 0;
+    const int tpp = p.bs / kTileTok;
+    const int first_tile = t0 / kTileTok;
+    const int32_t* table = p.block_tables + (size_t)s * p.max_blocks;
+    // Page ids of this warp's tiles, 32 at a time.  The index is held inside the table, so the loads do not depend on
+    // the sequence's length (they travel together with the load of n instead of after it; ids past the end are never
+    // used) and a length beyond max_blocks * bs gives a wrong row, not a stray access.
+    auto load_pages = [&](int kb) -> int {
+        return __ldg(table + min((first_tile + warp + (kb + lane) * kWarps) / tpp, p.max_blocks - 1));
+    };
+    int pages_cur = load_pages(0), pages_next = load_pages(32), blk = 0;
+    const int n = p.context_lens[s];
     const int t1 = split ? min(t0 + p.partition_size, n) : n;
 
     if (t0 >= t1) {
+        // Empty range.  The wait comes first all the same: an earlier kernel of the stream may still be reading out,
+        // and a grid none of whose CTAs waited could finish before its predecessor.
+        grid_dependency_wait();
         if (!split) {
             __nv_bfloat16* o = static_cast<__nv_bfloat16*>(p.out) + ((size_t)s * p.Hq + (size_t)kvh * G) * D;
             for (int e = threadIdx.x; e < G * D; e += blockDim.x) o[e] = __float2bfloat16_rn(0.f);
@@ -114,11 +133,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     float* lbuf = reinterpret_cast<float*>(smem + C::OFF_L);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR) + warp * kStages;
 
-    const int tpp = p.bs / kTileTok;
-    const int first_tile = t0 / kTileTok;
     const int ntiles = (t1 + kTileTok - 1) / kTileTok - first_tile;
     const int cnt = ntiles > warp ? (ntiles - warp + kWarps - 1) / kWarps : 0;
-    const int32_t* table = p.block_tables + (size_t)s * p.max_blocks;
 
     if (lane == 0) {
 #pragma unroll
@@ -127,12 +143,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     }
     __syncwarp();
 
-    auto load_pages = [&](int kb) -> int {
-        int k = kb + lane;
-        return k < cnt ? __ldg(table + (first_tile + warp + k * kWarps) / tpp) : 0;
-    };
-    int pages_cur = load_pages(0), pages_next = load_pages(32), blk = 0;
-
     auto issue = [&](int k) {
         if ((k >> 5) != blk) {
             pages_cur = pages_next;
@@ -140,6 +150,25 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             pages_next = load_pages((blk + 1) * 32);
         }
         const int phys = __shfl_sync(kFull, pages_cur, k & 31);
+        if (p.k_new && first_tile + warp + k * kWarps == (n - 1) / kTileTok) {
+            // The step's new token of this sequence lies in the tile about to be fetched (Algorithm 2, "Store reshaped
+            // K, V into C_K, C_V"): store its K and V rows of this head first, as the slot-mapped write would, and order
+            // the stores before the bulk copy.  The tile belongs to this warp alone, so nobody reads the row earlier.
+            const long long slot = __ldg(p.slot_mapping + s);
+            if (slot >= 0) {
+                constexpr int VEC = D * 2 / 16;                  // 16-byte vectors per row
+                if (lane < 2 * VEC) {
+                    const bool is_v = lane >= VEC;
+                    const int vi = lane % VEC;
+                    const size_t src = ((size_t)s * p.Hkv + kvh) * VEC + vi;
+                    const size_t dst = (((size_t)(slot / p.bs) * p.Hkv + kvh) * p.bs + (size_t)(slot % p.bs)) * VEC + vi;
+                    if (is_v) p.v_cache_w[dst] = __ldg(p.v_new + src);
+                    else p.k_cache_w[dst] = __ldg(p.k_new + src);
+                }
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+            }
+            __syncwarp();
+        }
         if (lane == 0) {
             const int tt = first_tile + warp + k * kWarps;
             const int row = (phys * p.Hkv + kvh) * p.bs + (tt % tpp) * kTileTok;   // row of the [rows, D] view
@@ -313,16 +342,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
 template <int D, int G, int kWarps, int kMinCtas>
 int launch_shape(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p, int B, cudaStream_t stream) {
     using C = TcCfg<D, G, kWarps>;
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
-    if (dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(decode_tc_kernel<D, G, kWarps, kMinCtas>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 C::SMEM) != cudaSuccess)
-            return OPT_GQA_ERR_CUDA;
-        configured[dev] = true;
-    }
-    dim3 grid(p.partition_size > 0 ? p.max_partitions : 1, p.Hkv, B);
+    static std::atomic<bool> configured[kMaxDevices];
+    if (!ensure_smem_limit(decode_tc_kernel<D, G, kWarps, kMinCtas>, C::SMEM, configured)) return OPT_GQA_ERR_CUDA;
+    const long long ctas = (long long)(p.partition_size > 0 ? p.max_partitions : 1) * p.Hkv * B;
+    if (ctas > 0x7fffffffll) return OPT_GQA_ERR_SHAPE;
+    dim3 grid((unsigned)ctas);
     return launch_dependent(decode_tc_kernel<D, G, kWarps, kMinCtas>, grid, dim3(kWarps * 32), C::SMEM, stream, mk, mv,
                             p);
 }
@@ -350,7 +374,7 @@ int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* 
                      int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                      int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
                      float* partial_out, float* partial_lse, int max_partitions, int* device_status,
-                     cudaStream_t stream) {
+                     cudaStream_t stream, const FusedAppend* append) {
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull) return OPT_GQA_ERR_SHAPE;
     CUtensorMap mk, mv;
@@ -372,6 +396,12 @@ int launch_decode_tc(void* out, const void* q, const void* k_cache, const void* 
     p.bs = bs;
     p.partition_size = partition_size;
     p.max_partitions = max_partitions;
+    p.B = B;
+    p.k_new = append ? static_cast<const uint4*>(append->k_new) : nullptr;
+    p.v_new = append ? static_cast<const uint4*>(append->v_new) : nullptr;
+    p.k_cache_w = append ? static_cast<uint4*>(append->k_cache) : nullptr;
+    p.v_cache_w = append ? static_cast<uint4*>(append->v_cache) : nullptr;
+    p.slot_mapping = append ? append->slot_mapping : nullptr;
     const int G = Hq / Hkv;
     if (D == 128) return launch_g<128>(mk, mv, p, B, G, stream);
     if (D == 64) return launch_g<64>(mk, mv, p, B, G, stream);

@@ -23,17 +23,19 @@ constexpr size_t kScratchFloats = OPT_GQA_STATIC_SCRATCH_BYTES / sizeof(float);
 // cudaGetSymbolAddress below.
 static __device__ __align__(256) float g_static_scratch[kScratchFloats];
 
-// Device address of the array on the current device, resolved once per device (with that device current).
+// Device address of the array on the current device, resolved once per device (with that device current; the
+// stream passed to the entry point must belong to that device).  The cache is atomic: host threads that make their
+// first call together each look the address up and store the same value.
 float* static_scratch_ptr() {
-    static float* ptrs[64] = {};
+    static std::atomic<float*> ptrs[kMaxDevices];
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ptrs[dev]) {
-        float* p = nullptr;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    float* p = ptrs[dev].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress((void**)&p, g_static_scratch) != cudaSuccess || !p) return nullptr;
-        ptrs[dev] = p;
+        ptrs[dev].store(p, std::memory_order_release);
     }
-    return ptrs[dev];
+    return p;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -52,7 +54,7 @@ extern "C" int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q,
                                                        void* stream) {
     if (dtype != OPT_GQA_FP32 && dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || (D != 64 && D != 128) || (bs != 16 && bs != 32) ||
-        max_blocks_per_seq < 0 || num_blocks < 0 || partition_size <= 0 || partition_size % 16 != 0 ||
+        max_blocks_per_seq < 0 || (B > 0 && max_blocks_per_seq == 0) || num_blocks < 0 || partition_size <= 0 || partition_size % 16 != 0 ||
         max_partitions <= 0)
         return OPT_GQA_ERR_SHAPE;
     const int G = Hq / Hkv;
@@ -78,8 +80,8 @@ extern "C" int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q,
                               partial_lse, max_partitions, status, cs);
     else
         rc = launch_decode(nullptr, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
-                           alibi_slopes, scale, B, Hq, Hkv, D, bs, partition_size, partial_out, partial_lse,
-                           max_partitions, dtype, status, cs);
+                           alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
+                           partial_lse, max_partitions, dtype, status, cs);
     if (rc != OPT_GQA_OK) return rc;
     return launch_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size, max_partitions,
                          dtype, cs);

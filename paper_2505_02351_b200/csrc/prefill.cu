@@ -84,7 +84,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const int qstart = p.q_start_loc[s];
     const int qlen = p.q_start_loc[s + 1] - qstart;
     const int nblk = (qlen + TQ - 1) / TQ;
-    if ((int)blockIdx.x >= nblk) return;
+    if ((int)blockIdx.x >= nblk) {
+        grid_dependency_wait();     // a grid none of whose CTAs waited could finish before its predecessor
+        return;
+    }
     const int qb = nblk - 1 - (int)blockIdx.x;             // the longest-running blocks start first
     const int n = p.context_lens[s];
     const int i_last = min(qlen, (qb + 1) * TQ) - 1;        // last valid new token of this block
@@ -316,14 +319,8 @@ template <int D, int G>
 int launch_one(const CUtensorMap& mk, const CUtensorMap& mv, const PrefillParams& p, int B, int max_q_len,
                cudaStream_t stream) {
     using C = PrefillCfg<D>;
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
-    if (dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(prefill_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
-            return OPT_GQA_ERR_CUDA;
-        configured[dev] = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];
+    if (!ensure_smem_limit(prefill_kernel<D, G>, C::SMEM, configured)) return OPT_GQA_ERR_CUDA;
     constexpr int TQ = kRows / G;
     dim3 grid((max_q_len + TQ - 1) / TQ, p.Hkv, B);
     return launch_dependent(prefill_kernel<D, G>, grid, dim3((kConsumers + 1) * 32), C::SMEM, stream, mk, mv, p);

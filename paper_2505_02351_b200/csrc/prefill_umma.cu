@@ -33,19 +33,10 @@ namespace {
 
 constexpr int kD = 128;            // head dimension
 constexpr int kRows = 128;         // rows of the CTA's tiles (G heads x TQ tokens)
-#ifndef OPT_GQA_PF_TN
-#define OPT_GQA_PF_TN 64
-#endif
-#ifndef OPT_GQA_PF_STAGES
-#define OPT_GQA_PF_STAGES 2
-#endif
-#ifndef OPT_GQA_PF_CTAS
-#define OPT_GQA_PF_CTAS 2
-#endif
-constexpr int kTN = OPT_GQA_PF_TN;  // keys per tile (64 or 128)
+constexpr int kTN = 64;            // keys per tile
 constexpr int kSub = 16;           // token rows per TMA box
-constexpr int kKvStages = OPT_GQA_PF_STAGES;
-constexpr int kCtasPerSm = OPT_GQA_PF_CTAS;
+constexpr int kKvStages = 2;
+constexpr int kCtasPerSm = 2;
 constexpr int kThreads = 192;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: O is rescaled only when a row's maximum grew by more
@@ -249,34 +240,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     return d;
 }
 
-#ifndef OPT_GQA_PF_POLY_PERIOD
-#define OPT_GQA_PF_POLY_PERIOD 0
-#endif
-// Every kPolyPeriod-th pair of a chunk takes 2^t from the FMA pipe instead of the special-function unit (0: none).
-constexpr int kPolyPeriod = OPT_GQA_PF_POLY_PERIOD;
-
-// 2^t for two values without the special-function unit: t = n + f with n = round(t) (taken from the low mantissa
-// bits of t + 1.5 * 2^23), 2^f on [-1/2, 1/2] by a cubic whose relative error (8e-5) is far below the bf16
-// rounding that follows, and n added to the exponent field.  t is clamped at -126: 2^-126 stands in for
-// anything smaller, masked keys included.
-__device__ __forceinline__ uint64_t exp2_pair_fma(uint64_t t2) {
-    float t0, t1;
-    unpack_f2(t2, t0, t1);
-    t2 = pack_f2(fmaxf(t0, -126.f), fmaxf(t1, -126.f));
-    const uint64_t magic = pack_f2(12582912.f, 12582912.f), neg_magic = pack_f2(-12582912.f, -12582912.f);
-    const uint64_t y2 = add2(t2, magic);
-    const uint64_t n2 = add2(y2, neg_magic);
-    const uint64_t f2 = fma2(n2, pack_f2(-1.f, -1.f), t2);
-    uint64_t r2 = fma2(pack_f2(0.05508868f, 0.05508868f), f2, pack_f2(0.24260405f, 0.24260405f));
-    r2 = fma2(r2, f2, pack_f2(0.69327623f, 0.69327623f));
-    r2 = fma2(r2, f2, pack_f2(0.99992895f, 0.99992895f));
-    float y0, y1, r0, r1;
-    unpack_f2(y2, y0, y1);
-    unpack_f2(r2, r0, r1);
-    return pack_f2(__int_as_float(__float_as_int(r0) + (__float_as_int(y0) << 23)),
-                   __int_as_float(__float_as_int(r1) + (__float_as_int(y1) << 23)));
-}
-
 // Pass 2 over one chunk: p = 2^(s*qscale + bias) with the tile's ALiBi constant and the row maximum folded into
 // bias; bf16 pairs for the tensor core; returns the chunk's sum of p.
 template <bool kMasked>
@@ -301,19 +264,10 @@ __device__ __forceinline__ float chunk_exp(const float (&v)[32], float qscale, f
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
         const uint64_t t2 = fma2(pack_f2(v[2 * e], v[2 * e + 1]), qs2, b2);
-        uint64_t p2;
-        float p0, p1;
-        if (kPolyPeriod > 0 && e % kPolyPeriod == kPolyPeriod - 1) {
-            p2 = exp2_pair_fma(t2);
-            unpack_f2(p2, p0, p1);
-        } else {
-            float t0, t1;
-            unpack_f2(t2, t0, t1);
-            p0 = ex2(t0);
-            p1 = ex2(t1);
-            p2 = pack_f2(p0, p1);
-        }
-        sm2[e & 1] = add2(sm2[e & 1], p2);
+        float t0, t1;
+        unpack_f2(t2, t0, t1);
+        const float p0 = ex2(t0), p1 = ex2(t1);
+        sm2[e & 1] = add2(sm2[e & 1], pack_f2(p0, p1));
         w[e] = pack2(p0, p1);
     }
     float s0, s1;
@@ -347,7 +301,10 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int qstart = p.q_start_loc[s];
     const int qlen = p.q_start_loc[s + 1] - qstart;
     const int nblk = (qlen + TQ - 1) / TQ;
-    if ((int)blockIdx.x >= nblk) return;
+    if ((int)blockIdx.x >= nblk) {
+        grid_dependency_wait();     // a grid none of whose CTAs waited could finish before its predecessor
+        return;
+    }
     const int qb = nblk - 1 - (int)blockIdx.x;             // the longest-running blocks start first
     const int n = kPaged ? p.context_lens[s] : qlen;
     const int i_last = min(qlen, (qb + 1) * TQ) - 1;        // last valid new token of this block
@@ -681,15 +638,8 @@ bool make_kv_map(CUtensorMap* map, const void* kv, int tokens, int Hkv) {
 template <int G, bool kPaged>
 int launch_one(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& p, int B,
                int max_q_len, cudaStream_t stream) {
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return OPT_GQA_ERR_CUDA;
-    if (dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(prefill_umma_kernel<G, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemBytes) != cudaSuccess)
-            return OPT_GQA_ERR_CUDA;
-        configured[dev] = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];
+    if (!ensure_smem_limit(prefill_umma_kernel<G, kPaged>, kSmemBytes, configured)) return OPT_GQA_ERR_CUDA;
     constexpr int TQ = kRows / G;
     dim3 grid((max_q_len + TQ - 1) / TQ, p.Hkv, B);
     return launch_dependent(prefill_umma_kernel<G, kPaged>, grid, dim3(kThreads), kSmemBytes, stream, mq, mk, mv, p);

@@ -3,21 +3,25 @@
 //   out = sum_p e^{lse_p - L} o_p / sum_p e^{lse_p - L},  L = max_p lse_p,  p < ceil(n_s / P).
 // One CTA per (sequence, query head).  A lane owns D/32 adjacent output columns, so a
 // warp reads one partial row as one coalesced segment; the warps of the CTA take the
-// partitions round-robin (independent loads in flight instead of one dependent chain
-// over all partitions) and are folded through shared memory at the end.
+// partitions round-robin and are folded through shared memory at the end.  The first
+// kReducePre rows of every warp's share are requested together with the log-sum-exps,
+// before the maximum is known (with up to 64 partitions that is all of them: the merge
+// is one round trip to memory, not two dependent ones).
 #include <type_traits>
 
 #include "common.cuh"
 
 namespace optgqa {
 
-constexpr int kReduceWarps = 4;
+constexpr int kReduceWarps = 8;
+constexpr int kReducePre = 8;
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kReduceWarps * 32)
 reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const float* __restrict__ partial_lse,
               const int32_t* __restrict__ context_lens, int Hq, int partition_size, int max_partitions) {
     constexpr int V = D / 32;             // columns per lane
+    using Vec = typename std::conditional<V == 4, float4, float2>::type;
     __shared__ float s_num[kReduceWarps][D];
     __shared__ float s_den[kReduceWarps];
     grid_dependency_launch();
@@ -25,7 +29,9 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
     const int s = row / Hq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n = context_lens[s];         // an input of the step, not produced by the decode grid
-    const int np = (n + partition_size - 1) / partition_size;
+    // never beyond the rows the decode grid had (max_partitions is the caller's promise; a length that breaks it gives
+    // a wrong row, not a read past the partials)
+    const int np = min((n + partition_size - 1) / partition_size, max_partitions);
     T* o = out + (size_t)row * D;
     grid_dependency_wait();                // the partials come from the decode grid; out may still be read by its last user
     if (np <= 0) {
@@ -35,6 +41,17 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
     const float* lse = partial_lse + (size_t)row * max_partitions;
     const float* po = partial_out + (size_t)row * max_partitions * D + lane * V;
 
+    float lpre[kReducePre];
+    Vec xpre[kReducePre];
+#pragma unroll
+    for (int k = 0; k < kReducePre; ++k) {
+        const int p = warp + k * kReduceWarps;
+        lpre[k] = -INFINITY;
+        if (p < np) {
+            lpre[k] = lse[p];
+            xpre[k] = *reinterpret_cast<const Vec*>(po + (size_t)p * D);
+        }
+    }
     float L = -INFINITY;
     for (int p = lane; p < np; p += 32) L = fmaxf(L, lse[p]);
 #pragma unroll
@@ -44,22 +61,22 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
 #pragma unroll
     for (int v = 0; v < V; ++v) num[v] = 0.f;
     float den = 0.f;
-#pragma unroll 4
-    for (int p = warp; p < np; p += kReduceWarps) {
-        const float w = ex2((lse[p] - L) * kLog2e);
+    auto add_row = [&](float l, Vec x) {
+        const float w = ex2((l - L) * kLog2e);
         den += w;
+        num[0] = fmaf(w, x.x, num[0]);
+        num[1] = fmaf(w, x.y, num[1]);
         if constexpr (V == 4) {
-            const float4 x = *reinterpret_cast<const float4*>(po + (size_t)p * D);
-            num[0] = fmaf(w, x.x, num[0]);
-            num[1] = fmaf(w, x.y, num[1]);
             num[2] = fmaf(w, x.z, num[2]);
             num[3] = fmaf(w, x.w, num[3]);
-        } else {
-            const float2 x = *reinterpret_cast<const float2*>(po + (size_t)p * D);
-            num[0] = fmaf(w, x.x, num[0]);
-            num[1] = fmaf(w, x.y, num[1]);
         }
-    }
+    };
+#pragma unroll
+    for (int k = 0; k < kReducePre; ++k)
+        if (warp + k * kReduceWarps < np) add_row(lpre[k], xpre[k]);
+#pragma unroll 4
+    for (int p = warp + kReducePre * kReduceWarps; p < np; p += kReduceWarps)
+        add_row(lse[p], *reinterpret_cast<const Vec*>(po + (size_t)p * D));
 #pragma unroll
     for (int v = 0; v < V; ++v) s_num[warp][lane * V + v] = num[v];
     if (lane == 0) s_den[warp] = den;

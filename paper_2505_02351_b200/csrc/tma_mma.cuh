@@ -79,7 +79,8 @@ using TensorMapEncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point query (no link against libcuda).
 inline TensorMapEncodeFn tensor_map_encode_fn() {
-    static TensorMapEncodeFn fn = nullptr;
+    static std::atomic<TensorMapEncodeFn> cached{nullptr};
+    TensorMapEncodeFn fn = cached.load(std::memory_order_acquire);
     if (!fn) {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
@@ -87,6 +88,7 @@ inline TensorMapEncodeFn tensor_map_encode_fn() {
             q != cudaDriverEntryPointSuccess)
             return nullptr;
         fn = reinterpret_cast<TensorMapEncodeFn>(p);
+        cached.store(fn, std::memory_order_release);
     }
     return fn;
 }

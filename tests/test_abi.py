@@ -69,3 +69,33 @@ def test_argument_checks_run_before_any_cuda_call(lib):
     assert r(one, one, one, one, 0, 4, 64, 16, 1, 0, null) == 0
     assert r(one, one, one, one, 1, 4, 64, 0, 1, 0, null) == -2
     assert r(null, one, one, one, 1, 4, 64, 16, 1, 0, null) == -1
+
+
+def test_undersized_workspace_is_a_host_side_error(lib):
+    """The calls that take a workspace take its size too and refuse one that is too small for the sizes given,
+    before any CUDA call (fake pointers are enough to see it)."""
+    one = ctypes.c_void_p(256)
+    B, Hq, Hkv, D, P, maxP = 8, 32, 4, 128, 512, 64
+    need = binding.workspace_bytes(B, Hq, D, maxP)
+    f = lib.opt_gqa_paged_attention_decode_balanced
+    assert f(one, one, one, one, 8, one, one, 1.0, B, Hq, Hkv, D, 16, 100, P, one, need // 2, maxP, 1, None) == -2
+    assert f(one, one, one, one, 8, one, one, 1.0, B, Hq, Hkv, D, 16, 100, P, one, 0, maxP, 1, None) == -2
+    r = lib.opt_gqa_paged_attention_reduce_balanced
+    assert r(one, one, need // 2, one, B, Hq, Hkv, D, P, maxP, 1, None) == -2
+    loc = lib.opt_gqa_paged_attention_decode_local
+    assert loc(one, one, one, one, one, 8, one, one, 1.0, B, Hq, Hkv, D, 16, 100, P, one, 1024, maxP, 100, 1, None) == -2
+    st = lib.opt_gqa_decode_step
+    assert st(one, one, one, one, one, one, one, one, 8, one, one, 1.0, B, Hq, Hkv, D, 16, 100, P, one, need // 2, maxP, 1,
+              None) == -2
+    # fp32 caches: one (D + 1)-float row per (sequence, head, partition)
+    assert st(one, one, one, one, one, one, one, one, 8, one, one, 1.0, B, Hq, Hkv, D, 16, 100, P, one,
+              B * Hq * maxP * (D + 1) * 4 - 4, maxP, 0, None) == -2
+
+
+def test_debug_entry_points_check_their_arguments(lib):
+    assert lib.opt_gqa_debug_wait_timeout(0, None) == -2
+    assert lib.opt_gqa_debug_wait_timeout(1 << 25, None) == -2
+    assert lib.opt_gqa_debug_read_stream(None, 0, None, None) == 0
+    assert lib.opt_gqa_debug_read_stream(None, 8192, None, None) == -1
+    assert lib.opt_gqa_debug_read_stream(ctypes.c_void_p(256), 100, ctypes.c_void_p(256), None) == -2
+    assert lib.opt_gqa_debug_read_stream(ctypes.c_void_p(8), 8192, ctypes.c_void_p(256), None) == -4

@@ -317,3 +317,136 @@ def test_host_step_called_repeatedly_reads_the_buffers_anew():
         assert binding.device_status() == 0
         want = util.oracle_attention(W.Workload(**{**wl.__dict__, "q": q}))
         assert np.max(np.abs(hout.double().numpy() - want)) <= util.TOL["bf16"], call
+
+
+@pytest.mark.parametrize("shape", [(32, 4, 128, 16), (8, 2, 64, 32), (4, 4, 128, 32)])
+def test_bf16_partials_of_the_tile_kernel_match_the_oracle_partials(shape):
+    """opt_gqa_paged_attention_decode on bf16 caches (the tensor-core tile kernel, one CTA per partition): every
+    partition's normalised result and log-sum-exp on their own, not only the merged output."""
+    import oracle
+    Hq, Hkv, D, bs = shape
+    P = 64
+    wl = W.make_custom("pbf16", "bf16", Hq, Hkv, D, bs, [130, 40, 77, 1, 0, 1029], seed=61, poison=True)
+    _, d = util.gpu_decode(wl, partition_size=P)
+    a = util.oracle_inputs(wl)
+    maxP = d.partial_out.shape[2]
+    po, pl = oracle.partition_partials(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"], wl.scale, wl.dtype, P, maxP)
+    gpo, gpl = d.partial_out.double().cpu().numpy(), d.partial_lse.double().cpu().numpy()
+    for s in range(wl.B):
+        np_s = (int(a["n"][s]) + P - 1) // P
+        # p enters the tensor core rounded to bf16 (relative 2^-9 per term, averaged by the normalised sum)
+        assert np.max(np.abs(gpo[s, :, :np_s] - po[s, :, :np_s]), initial=0.0) <= util.TOL["bf16"]
+        assert np.max(np.abs(gpl[s, :, :np_s] - pl[s, :, :np_s]), initial=0.0) <= 5e-3
+        assert np.isnan(gpo[s, :, np_s:]).all() and np.isnan(gpl[s, :, np_s:]).all()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("D", [64, 128])
+def test_reduce_kernel_alone_on_the_oracle_partials(dtype, D):
+    """opt_gqa_paged_attention_reduce fed with the ORACLE's partials (rounded to fp32) against the oracle's merge:
+    the merge kernel on its own, with no decode kernel of the library in the loop."""
+    import oracle
+    P = 32
+    wl = W.make_custom("ronly", dtype, 8, 2, D, 16, [700, 33, 0, 31, 32, 2049], seed=62)
+    a = util.oracle_inputs(wl)
+    maxP = (2049 + P - 1) // P
+    po, pl = oracle.partition_partials(a["q"], a["k"], a["v"], a["bt"], a["n"], a["slopes"], wl.scale, wl.dtype, P, maxP)
+    po32, pl32 = po.astype(np.float32), pl.astype(np.float32)
+    for s in range(wl.B):                   # entries past a sequence's partitions must never be read
+        np_s = (int(a["n"][s]) + P - 1) // P
+        po32[s, :, np_s:] = np.nan
+        pl32[s, :, np_s:] = np.nan
+    want = oracle.reduce(po32.astype(np.float64), pl32.astype(np.float64), a["n"], P)
+    out = torch.full((wl.B, wl.Hq, D), float("nan"), device="cuda:0", dtype=W.TORCH_DTYPES[dtype])
+    binding.paged_attention_reduce(out, torch.from_numpy(po32).cuda(), torch.from_numpy(pl32).cuda(),
+                                   wl.context_lens.cuda(), P)
+    torch.cuda.synchronize()
+    got = out.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.max(np.abs(got - want)) <= (1e-6 if dtype == "fp32" else 2.0 ** -8 * 4.5)   # fp32 sums; one bf16 rounding
+    assert np.array_equal(got[2], np.zeros_like(got[2]))                                    # the empty sequence
+
+
+@pytest.mark.parametrize("dtype,simt", [("fp32", False), ("bf16", False), ("bf16", True)])
+def test_context_lengths_beyond_the_promised_sizes_stay_inside_the_buffers(dtype, simt):
+    """A length that breaks the caller's promises (n_s > max_partitions * P, n_s > max_blocks * bs) must give a wrong
+    row for that sequence, never an access outside the page table, the pool or the partials: canary rows around the
+    partials stay intact and the other sequences keep their results."""
+    wl = W.make_custom("promise", dtype, 8, 2, 128, 16, [100, 300, 64], seed=63)
+    d = util.DeviceWorkload(wl)
+    binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
+    want = util.oracle_attention(wl)
+    P, maxP = 64, 5
+    lens = wl.context_lens.clone()
+    lens[1] = 300 + 64 * 40                         # far past max_partitions * P and past the page table
+    rows = wl.B * wl.Hq * maxP
+    po = torch.full((rows + 2 * wl.Hq, wl.D), 7.0, device="cuda:0", dtype=torch.float32)   # canaries before and after
+    pl = torch.full((rows + 2 * wl.Hq,), 7.0, device="cuda:0", dtype=torch.float32)
+    po_in = po[wl.Hq: wl.Hq + rows].view(wl.B, wl.Hq, maxP, wl.D)
+    pl_in = pl[wl.Hq: wl.Hq + rows].view(wl.B, wl.Hq, maxP)
+    decode = binding.paged_attention_decode_simt if simt else binding.paged_attention_decode
+    decode(None, d.q, d.k_cache, d.v_cache, d.block_tables, lens.cuda(), d.alibi_slopes, wl.scale, partition_size=P,
+           partial_out=po_in, partial_lse=pl_in, max_partitions=maxP)
+    binding.paged_attention_reduce(d.out, po_in, pl_in, lens.cuda(), P)
+    decode(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, lens.cuda(), d.alibi_slopes, wl.scale)   # single pass too
+    binding.paged_attention_reduce(d.out, po_in, pl_in, lens.cuda(), P)
+    torch.cuda.synchronize()
+    assert binding.device_status() == 0
+    assert bool((po[: wl.Hq] == 7.0).all()) and bool((po[wl.Hq + rows:] == 7.0).all())
+    assert bool((pl[: wl.Hq] == 7.0).all()) and bool((pl[wl.Hq + rows:] == 7.0).all())
+    got = d.out.double().cpu().numpy()
+    for s in (0, 2):
+        assert np.max(np.abs(got[s] - want[s])) <= util.TOL[dtype]
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    """Failure detection without a fault: one warp waits, with a short limit, for bytes nobody sends; the kernel
+    records the timeout in the status word and returns.  The status reads -6 once, then 0, and decode still works."""
+    assert binding.device_status() == 0
+    binding.debug_wait_timeout(1 << 16)
+    torch.cuda.synchronize()
+    assert binding.device_status() == -6
+    assert binding.status_string(-6) == "a bounded device-side wait ran out"
+    assert binding.device_status() == 0
+    with pytest.raises(binding.OptGqaError):
+        binding.debug_wait_timeout(1 << 30)          # limits are capped: no long waits on request
+    wl = W.make_custom("after", "bf16", 8, 2, 128, 16, [700, 33], seed=64)
+    _check(wl, partition_size=256, balanced=True)
+    _check(wl)
+
+
+def test_read_stream_probe_reads_every_chunk():
+    """The read-only probe of the benchmark: its checksum is the XOR of one 16-byte word per 256 bytes."""
+    n = 8192 * 301
+    src = torch.randint(-2**31, 2**31 - 1, (n // 4,), dtype=torch.int32, device="cuda:0")
+    chk = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    binding.debug_read_stream(src, chk)
+    torch.cuda.synchronize()
+    assert binding.device_status() == 0
+    words = src.cpu().numpy().view(np.uint32).reshape(-1, 64)[:, :4]       # the first 16 bytes of every 256
+    assert int(chk.cpu().numpy().view(np.uint32)[0]) == int(np.bitwise_xor.reduce(words.reshape(-1)))
+
+
+def test_undersized_workspace_is_refused_before_anything_runs():
+    wl = W.make_custom("ws", "bf16", 8, 2, 128, 16, [700, 33], seed=65)
+    d = util.DeviceWorkload(wl)
+    P, maxP = 64, 11
+    need = binding.workspace_bytes(wl.B, wl.Hq, wl.D, maxP)
+    small = torch.empty(need // 2, dtype=torch.uint8, device="cuda:0")
+    d.out.fill_(3.0)
+    for call in (
+        lambda: binding.paged_attention_decode_balanced(d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+                                                        d.alibi_slopes, wl.scale, P, small, maxP),
+        lambda: binding.paged_attention_reduce_balanced(d.out, small, d.context_lens, wl.Hkv, P, maxP),
+        lambda: binding.paged_attention_decode_local(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+                                                     d.alibi_slopes, wl.scale, P, small, maxP, 100),
+        lambda: binding.decode_step(d.out, d.q, d.k_new, d.v_new, d.slot_mapping, d.k_cache, d.v_cache, d.block_tables,
+                                    d.context_lens, d.alibi_slopes, wl.scale, partition_size=P, workspace=small,
+                                    max_partitions=maxP),
+    ):
+        with pytest.raises(binding.OptGqaError) as e:
+            call()
+        assert e.value.code == -2
+    torch.cuda.synchronize()
+    assert bool((d.out == 3.0).all())
+    assert torch.equal(d.k_cache.cpu(), wl.k_cache)        # the fused append did not run either

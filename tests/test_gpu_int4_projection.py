@@ -113,3 +113,48 @@ def test_projection_rejects_bad_arguments():
     assert binding.int4_packed_bytes(512, 768, 128) == 512 * 768 // 2 + 4 * 768 * 4
     assert binding.int4_packed_bytes(512, 760, 128) == 0
     torch.cuda.synchronize()
+
+
+def test_projection_then_decode_on_one_stream_without_synchronisation():
+    """Eq. 1 -> "Reshape and store K, V" -> "Compute context attention with caches" as one chain on one stream: the
+    projection lets its dependents start early and writes q and the new K/V rows; the balanced decode and its merge
+    must see them (q is read only after the dependency wait, through L2).  Repeated with new activations into the
+    same buffers, so that a stale line of the previous round's q would show."""
+    from tests import util
+
+    Hq, Hkv, D, K, gs = 32, 4, 128, 4096, 128
+    wl = W.make_custom("chain", "bf16", Hq, Hkv, D, 16, [3000, 1500, 700, 2049, 16, 1, 512, 4000], seed=81)
+    d = util.DeviceWorkload(wl)
+    T, N = wl.B, (Hq + 2 * Hkv) * D
+    p = W.make_int4_projection(82, T, K, N, gs)
+    packed = torch.empty(binding.int4_packed_bytes(K, N, gs), dtype=torch.uint8, device=DEV)
+    binding.int4_prepack(packed, p.qweight.to(DEV), p.scales.to(DEV), p.qzeros.to(DEV), gs)
+    P, maxP = 512, 8
+    ws = torch.empty(binding.workspace_bytes(wl.B, Hq, D, maxP), dtype=torch.uint8, device=DEV)
+    q_buf = torch.zeros((T, Hq, D), dtype=torch.bfloat16, device=DEV)
+    gen = torch.Generator().manual_seed(83)
+    stream = torch.cuda.Stream()
+    for rep in range(4):
+        x = (0.3 * torch.randn((T, K), generator=gen)).to(torch.bfloat16).to(DEV)
+        d.out.fill_(float("nan"))
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            binding.qkv_project_int4(q_buf, x, packed, Hq, Hkv, D, gs, k_cache=d.k_cache, v_cache=d.v_cache,
+                                     slot_mapping=d.slot_mapping)
+            binding.paged_attention_decode_balanced(q_buf, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+                                                    d.alibi_slopes, wl.scale, P, ws, maxP)
+            binding.paged_attention_reduce_balanced(d.out, ws, d.context_lens, Hkv, P, maxP)
+        stream.synchronize()
+        assert binding.device_status() == 0
+        # the oracle attends with the projection's own outputs (read back after the chain has finished)
+        want = oracle.paged_attention(W.storage_numpy(q_buf), W.storage_numpy(d.k_cache), W.storage_numpy(d.v_cache),
+                                      wl.block_tables.numpy(), wl.context_lens.numpy(),
+                                      wl.alibi_slopes.numpy().astype(np.float64), wl.scale, "bf16")
+        got = d.out.double().cpu().numpy()
+        assert np.isfinite(got).all()
+        assert np.max(np.abs(got - want)) <= util.TOL["bf16"], rep
+        # and q is what Eq. 1 gives for this round's activations
+        y = oracle.qkv_project_int4(W.storage_numpy(x), p.qweight.numpy().view(np.uint32), W.storage_numpy(p.scales),
+                                    p.qzeros.numpy().view(np.uint32), gs)
+        got_q = q_buf.double().cpu().numpy().reshape(T, Hq * D)
+        assert np.all(np.abs(got_q - y[:, :Hq * D]) <= _tol(y[:, :Hq * D]))

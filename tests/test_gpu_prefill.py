@@ -94,10 +94,22 @@ def test_empty_sequences_and_no_new_tokens():
     _check(wl)
 
 
-def test_config5_full_size_sampled_rows():
-    """The full workload in the configuration the benchmark times; the oracle checks sampled rows one by one."""
+def test_config5_full_size_every_row():
+    """The full workload in the configuration the benchmark times (a query block sees up to 96 key tiles), every one
+    of its 8192 x 32 output rows against the oracle (about half a minute of fp64 on the host cores)."""
     wl = W.make_config(5)
     got, _ = util.gpu_prefill(wl)
+    assert np.isfinite(got).all()
+    want = util.oracle_attention(wl)
+    assert got.shape == want.shape == (4 * 2048, 32, 128)
+    err = np.max(np.abs(got - want))
+    assert err <= TOL, err
+
+
+def test_config5_full_size_on_the_warp_level_kernel_sampled_rows():
+    """The same workload through opt_gqa_paged_attention_prefill_mma; the oracle checks sampled rows one by one."""
+    wl = W.make_config(5)
+    got, _ = util.gpu_prefill(wl, mma=True)
     assert np.isfinite(got).all()
     rng = np.random.default_rng(5)
     rows = np.unique(np.concatenate([rng.integers(0, wl.T, size=24), [0, 2047, 2048, wl.T - 1]]))
