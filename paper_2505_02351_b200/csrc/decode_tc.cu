@@ -97,9 +97,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     grid_dependency_launch();   // the grid after this one (the reduce) may start its own prologue
     const uint64_t read_once = l2_policy_evict_first();     // every K/V byte is read exactly once
     const uint64_t keep = l2_policy_evict_last();           // the partial results are read by the merge that follows
-    // Work item of this CTA.  The sequence index runs fastest and the partition index slowest, so that the grid ends
-    // with the high partition numbers, which only the longest sequences have: the last CTAs to start are few and short.
-    const int s = blockIdx.x % p.B, kvh = (blockIdx.x / p.B) % p.Hkv, part = blockIdx.x / (p.B * p.Hkv);
+    // Work item of this CTA.  The KV head runs fastest: CTAs that start together read the same pages (a page holds the
+    // rows of all KV heads side by side), which keeps the DRAM accesses of a moment close together.  The partition
+    // index runs slowest, so that the grid ends with the high partition numbers, which only the longest sequences
+    // have: the last CTAs to start are few and short.
+    const int kvh = blockIdx.x % p.Hkv, s = (blockIdx.x / p.Hkv) % p.B, part = blockIdx.x / (p.B * p.Hkv);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;      // fragment row (query head of the group) and column pair
     const bool split = p.partition_size > 0;
