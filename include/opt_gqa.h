@@ -226,8 +226,8 @@ int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q, const void
  *   q_start_loc   [B+1] int32              prefix sums of q_len_s, device memory
  *   total_q_tokens HOST value: rows of q and out (= q_start_loc[B]); rows are read up to it
  *   max_q_len     HOST value >= max_s q_len_s (sizes the grid)
- * D = 128 with scale > 0 runs on tcgen05.mma with accumulators in tensor memory; D = 64, or a
- * scale that is not positive, on warp-level mma.
+ * Runs on tcgen05.mma with accumulators in tensor memory, for both head dimensions and any scale (a
+ * negative scale negates Q inside the instruction, a zero scale leaves the dot products out).
  */
 int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
                                     int max_q_len, const void* k_cache, const void* v_cache,
@@ -238,7 +238,7 @@ int opt_gqa_paged_attention_prefill(void* out, const void* q, const int32_t* q_s
 /*
  * The same operation, arguments and results as opt_gqa_paged_attention_prefill, forced onto the
  * warp-level kernel (mma.sync m16n8k16, eight consumer warps of 16 rows each and a producer warp):
- * keeps the earlier form of Eq. 3-5 reachable for D = 128 as a cross-check and for comparison.
+ * keeps the earlier form of Eq. 3-5 reachable as a cross-check and for comparison.
  */
 int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens,
                                         int max_q_len, const void* k_cache, const void* v_cache,
@@ -254,10 +254,14 @@ int opt_gqa_paged_attention_prefill_mma(void* out, const void* q, const int32_t*
  * a sequence's stream (or a query block's key range) starts at, and the edge tile is masked from the
  * indices.
  *
- * opt_gqa_paged_attention_decode_local: the balanced split and its merge in one call (arguments as
- * opt_gqa_paged_attention_decode_balanced followed by opt_gqa_paged_attention_reduce_balanced; out
- * [B, Hq, D] is written; bf16 caches, partition_size > 0).  opt_gqa_paged_attention_prefill_local:
- * arguments as opt_gqa_paged_attention_prefill (bf16, D = 128, scale > 0).  window > 0 is required.
+ * opt_gqa_paged_attention_decode_local: split decode and merge in one call, out [B, Hq, D] is written,
+ * partition_size > 0.  bf16 caches take the balanced split (arguments as
+ * opt_gqa_paged_attention_decode_balanced followed by opt_gqa_paged_attention_reduce_balanced); fp32 caches
+ * one partial per partition on the CUDA-core kernel, partial_out [B, Hq, max_partitions, D] followed by
+ * partial_lse at the start of the workspace (workspace_bytes >= B * Hq * max_partitions * (D + 1) * 4),
+ * and the merge skips the partitions that lie wholly before the window.
+ * opt_gqa_paged_attention_prefill_local: arguments as opt_gqa_paged_attention_prefill (bf16).
+ * window > 0 is required.
  */
 int opt_gqa_paged_attention_decode_local(void* out, const void* q, const void* k_cache, const void* v_cache,
                                          const int32_t* block_tables, int max_blocks_per_seq,
@@ -278,11 +282,11 @@ int opt_gqa_paged_attention_prefill_local(void* out, const void* q, const int32_
  * for GQA grouping", "Create ALiBi bias", then Eq. 3-5): every sequence attends causally to its own
  * new tokens, read from contiguous tensors instead of the paged cache.  Token i of sequence s
  * (row q_start_loc[s] + i) sees keys 0 .. i of that sequence with bias -slope_h*(i - j); query
- * head h uses K/V head h / G.  The same tcgen05 kernel as opt_gqa_paged_attention_prefill, with
- * K/V tiles fetched through 3-D tensor maps over k and v.  (Writing k, v into the cache for later
+ * head h uses K/V head h / G.  The same tcgen05 kernel as opt_gqa_paged_attention_prefill (D 64 or 128,
+ * any scale), with K/V tiles fetched through 3-D tensor maps over k and v.  (Writing k, v into the cache for later
  * decode steps is opt_gqa_cache_append, before or after this call.)
  *
- *   out, q        [total_q_tokens, Hq, D]   bf16, D = 128
+ *   out, q        [total_q_tokens, Hq, D]   bf16
  *   k, v          [total_q_tokens, Hkv, D]  bf16
  *   q_start_loc   [B+1] int32               prefix sums of the sequences' lengths, device memory
  *   total_q_tokens, max_q_len               HOST values, as in opt_gqa_paged_attention_prefill

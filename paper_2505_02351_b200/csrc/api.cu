@@ -52,7 +52,7 @@ int opt_gqa_cache_append(const void* k_new, const void* v_new, void* k_cache, vo
                                static_cast<cudaStream_t>(stream));
 }
 
-static int decode_checked(bool allow_tensor_cores, void* out, const void* q, const void* k_cache, const void* v_cache,
+static int decode_checked(bool allow_tensor_cores, int window, void* out, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* block_tables, int max_blocks_per_seq, const int32_t* context_lens,
                           const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D, int bs,
                           int64_t num_blocks, int partition_size, float* partial_out, float* partial_lse,
@@ -85,7 +85,7 @@ static int decode_checked(bool allow_tensor_cores, void* out, const void* q, con
                                 partial_lse, max_partitions, status, cs);
     return launch_decode(out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
                          scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out, partial_lse, max_partitions,
-                         dtype, status, cs);
+                         window, dtype, status, cs);
 }
 
 int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache, const void* v_cache,
@@ -94,7 +94,7 @@ int opt_gqa_paged_attention_decode(void* out, const void* q, const void* k_cache
                                    int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
                                    float* partial_out, float* partial_lse, int max_partitions, int dtype,
                                    void* stream) {
-    return decode_checked(true, out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+    return decode_checked(true, 0, out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                           alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
                           partial_lse, max_partitions, dtype, stream);
 }
@@ -105,7 +105,7 @@ int opt_gqa_paged_attention_decode_simt(void* out, const void* q, const void* k_
                                         int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size,
                                         float* partial_out, float* partial_lse, int max_partitions, int dtype,
                                         void* stream) {
-    return decode_checked(false, out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+    return decode_checked(false, 0, out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                           alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
                           partial_lse, max_partitions, dtype, stream);
 }
@@ -120,7 +120,7 @@ int opt_gqa_paged_attention_reduce(void* out, const float* partial_out, const fl
     if (B == 0) return OPT_GQA_OK;
     if (!out || !partial_out || !partial_lse || !context_lens) return OPT_GQA_ERR_NULL;
     if (!aligned16(out) || !aligned16(partial_out)) return OPT_GQA_ERR_ALIGN;
-    return launch_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size, max_partitions,
+    return launch_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size, max_partitions, 0,
                          dtype, static_cast<cudaStream_t>(stream));
 }
 
@@ -189,6 +189,24 @@ int opt_gqa_paged_attention_decode_local(void* out, const void* q, const void* k
                                          int dtype, void* stream) {
     if (window <= 0) return OPT_GQA_ERR_SHAPE;
     if (B > 0 && !out) return OPT_GQA_ERR_NULL;
+    if (dtype == OPT_GQA_FP32) {
+        // fp32 caches: one partial per partition on the CUDA-core kernel (partial_out followed by partial_lse at
+        // the start of the workspace), then the merge over the partitions that hold attended keys
+        if (B < 0 || partition_size <= 0 || max_partitions <= 0 || Hq <= 0 || D <= 0) return OPT_GQA_ERR_SHAPE;
+        if (B == 0) return OPT_GQA_OK;
+        if (!workspace) return OPT_GQA_ERR_NULL;
+        const size_t rows = (size_t)B * Hq * max_partitions;
+        if (workspace_bytes < rows * ((size_t)D + 1) * 4) return OPT_GQA_ERR_SHAPE;
+        if (!aligned16(out) || !aligned16(workspace)) return OPT_GQA_ERR_ALIGN;
+        float* partial_out = static_cast<float*>(workspace);
+        float* partial_lse = partial_out + rows * D;
+        int rc = decode_checked(false, window, out, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
+                                alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
+                                partial_lse, max_partitions, dtype, stream);
+        if (rc != OPT_GQA_OK) return rc;
+        return launch_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size, max_partitions,
+                             window, dtype, static_cast<cudaStream_t>(stream));
+    }
     int rc = decode_balanced_checked(q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens, alibi_slopes,
                                      scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, workspace, workspace_bytes,
                                      max_partitions, window, dtype, stream);
@@ -205,7 +223,7 @@ static int prefill_checked(bool allow_umma, int window, void* out, const void* q
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0 ||
-        num_blocks < 0 || window < 0 || (window > 0 && !(allow_umma && D == 128)))
+        num_blocks < 0 || window < 0 || (window > 0 && !allow_umma))
         return OPT_GQA_ERR_SHAPE;
     if (B == 0 || max_q_len == 0 || total_q_tokens == 0) return OPT_GQA_OK;
     if (num_blocks == 0) return OPT_GQA_ERR_SHAPE;
@@ -213,11 +231,9 @@ static int prefill_checked(bool allow_umma, int window, void* out, const void* q
     if (!aligned16(out) || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return OPT_GQA_ERR_ALIGN;
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
-    // the tcgen05 kernel folds scale into its score tile and needs it positive; anything else takes the other kernel
-    if (window > 0 && !(scale > 0.f)) return OPT_GQA_ERR_SHAPE;
-    if (allow_umma && D == 128 && scale > 0.f)
+    if (allow_umma)
         return launch_prefill_umma(out, q, q_start_loc, total_q_tokens, max_q_len, k_cache, v_cache, block_tables,
-                                   max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, bs, num_blocks,
+                                   max_blocks_per_seq, context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks,
                                    window, status, static_cast<cudaStream_t>(stream));
     return launch_prefill(out, q, q_start_loc, max_q_len, k_cache, v_cache, block_tables, max_blocks_per_seq,
                           context_lens, alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, status,
@@ -261,14 +277,13 @@ int opt_gqa_prompt_attention(void* out, const void* q, const void* k, const void
                              int Hkv, int D, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (dtype != OPT_GQA_BF16) return OPT_GQA_ERR_DTYPE;
-    if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, 16) || D != 128 || !(scale > 0.f))
-        return OPT_GQA_ERR_SHAPE;
+    if (B < 0 || max_q_len < 0 || total_q_tokens < 0 || !shape_ok(Hq, Hkv, D, 16)) return OPT_GQA_ERR_SHAPE;
     if (B == 0 || max_q_len == 0 || total_q_tokens == 0) return OPT_GQA_OK;
     if (!out || !q || !k || !v || !q_start_loc) return OPT_GQA_ERR_NULL;
     if (!aligned16(out) || !aligned16(q) || !aligned16(k) || !aligned16(v)) return OPT_GQA_ERR_ALIGN;
     int* status = device_status_ptr();
     if (!status) return OPT_GQA_ERR_CUDA;
-    return launch_prompt_umma(out, q, k, v, q_start_loc, total_q_tokens, max_q_len, alibi_slopes, scale, B, Hq, Hkv,
+    return launch_prompt_umma(out, q, k, v, q_start_loc, total_q_tokens, max_q_len, alibi_slopes, scale, B, Hq, Hkv, D,
                               status, static_cast<cudaStream_t>(stream));
 }
 

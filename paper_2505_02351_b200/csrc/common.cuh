@@ -195,7 +195,8 @@ int launch_cache_append(const void* k_new, const void* v_new, void* k_cache, voi
 int launch_decode(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                   int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                   int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size, float* partial_out,
-                  float* partial_lse, int max_partitions, int dtype, int* device_status, cudaStream_t stream);
+                  float* partial_lse, int max_partitions, int window, int dtype, int* device_status,
+                  cudaStream_t stream);
 
 // Workspace of the balanced split (bf16 caches, partition_size > 0).  The stream of 16-token tiles
 // (sequence, KV head, partition order) is cut into one range per worker at TILE granularity; a piece is the
@@ -254,23 +255,25 @@ long long stream_grid_workers(int B, int Hkv, int max_partitions, int partition_
 int launch_reduce_balanced(void* out, const void* workspace, const int32_t* context_lens, int B, int Hq, int Hkv,
                            int D, int partition_size, int max_partitions, int window, int dtype, cudaStream_t stream);
 
+// window > 0: the partitions that lie wholly before a sequence's last `window` keys were not written and are skipped.
 int launch_reduce(void* out, const float* partial_out, const float* partial_lse, const int32_t* context_lens,
-                  int B, int Hq, int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream);
+                  int B, int Hq, int D, int partition_size, int max_partitions, int window, int dtype,
+                  cudaStream_t stream);
 
 int launch_prefill(void* out, const void* q, const int32_t* q_start_loc, int max_q_len, const void* k_cache,
                    const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
                    const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
                    int D, int bs, int64_t num_blocks, int* device_status, cudaStream_t stream);
 
-// bf16, D = 128: tcgen05.mma with accumulators in tensor memory (prefill_umma.cu).
+// bf16, any scale: tcgen05.mma with accumulators in tensor memory (prefill_umma.cu).
 int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens, int max_q_len,
                         const void* k_cache, const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
-                        int bs, int64_t num_blocks, int window, int* device_status, cudaStream_t stream);
+                        int D, int bs, int64_t num_blocks, int window, int* device_status, cudaStream_t stream);
 
-// bf16, D = 128: the prompt branch with empty caches (contiguous k, v of the new tokens), same kernel.
+// bf16: the prompt branch with empty caches (contiguous k, v of the new tokens), same kernel.
 int launch_prompt_umma(void* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,
                        int total_q_tokens, int max_q_len, const float* alibi_slopes, float scale, int B, int Hq,
-                       int Hkv, int* device_status, cudaStream_t stream);
+                       int Hkv, int D, int* device_status, cudaStream_t stream);
 
 }  // namespace optgqa

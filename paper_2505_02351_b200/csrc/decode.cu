@@ -38,6 +38,7 @@ struct DecodeParams {
     int bs;
     int partition_size;
     int max_partitions;
+    int window;             // > 0: only the last `window` keys of each sequence are attended to
 };
 
 constexpr int kTileTok = 16;   // tokens per tile (one ring stage holds a K tile and a V tile)
@@ -145,8 +146,9 @@ decode_kernel(const DecodeParams p) {
     const int half = lane >> 4, c = lane & 15;
     const int n = p.context_lens[s];
     const bool split = p.partition_size > 0;
-    const int t0 = split ? part * p.partition_size : 0;
-    const int t1 = split ? min(t0 + p.partition_size, n) : n;
+    const int start = p.window > 0 ? max(0, n - p.window) : 0;     // first attended key (local mask)
+    const int t0 = max(split ? part * p.partition_size : 0, start);
+    const int t1 = split ? min((part + 1) * p.partition_size, n) : n;
 
     if (t0 >= t1) {
         // Empty range.  A single-pass call still owes zero rows for an empty sequence.  The wait comes first all the
@@ -276,7 +278,7 @@ decode_kernel(const DecodeParams p) {
             float v = reduce_heads<G>(a);
             const int j = j0 + r;
             v = fmaf(slope2, (float)(j - (n - 1)), v);
-            sc[i] = j < t1 ? v : -INFINITY;
+            sc[i] = (j < t1 && j >= t0) ? v : -INFINITY;
         }
 
         // ---- online softmax update (per head, shared by both half-warps)
@@ -401,7 +403,8 @@ static int launch_g(const DecodeParams& p, int B, int G, cudaStream_t stream) {
 int launch_decode(void* out, const void* q, const void* k_cache, const void* v_cache, const int32_t* block_tables,
                   int max_blocks_per_seq, const int32_t* context_lens, const float* alibi_slopes, float scale,
                   int B, int Hq, int Hkv, int D, int bs, int64_t num_blocks, int partition_size, float* partial_out,
-                  float* partial_lse, int max_partitions, int dtype, int* device_status, cudaStream_t stream) {
+                  float* partial_lse, int max_partitions, int window, int dtype, int* device_status,
+                  cudaStream_t stream) {
     if (num_blocks <= 0 || num_blocks > 0x7fffffffll) return OPT_GQA_ERR_SHAPE;
     DecodeParams p;
     p.num_blocks = (int)num_blocks;
@@ -422,6 +425,7 @@ int launch_decode(void* out, const void* q, const void* k_cache, const void* v_c
     p.bs = bs;
     p.partition_size = partition_size;
     p.max_partitions = max_partitions;
+    p.window = window;
     const int G = Hq / Hkv;
     if (dtype == OPT_GQA_BF16) {
         if (D == 128) return launch_g<__nv_bfloat16, 128>(p, B, G, stream);

@@ -81,8 +81,8 @@ extern "C" int opt_gqa_paged_attention_decode_no_alloc(void* out, const void* q,
     else
         rc = launch_decode(nullptr, q, k_cache, v_cache, block_tables, max_blocks_per_seq, context_lens,
                            alibi_slopes, scale, B, Hq, Hkv, D, bs, num_blocks, partition_size, partial_out,
-                           partial_lse, max_partitions, dtype, status, cs);
+                           partial_lse, max_partitions, 0, dtype, status, cs);
     if (rc != OPT_GQA_OK) return rc;
-    return launch_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size, max_partitions,
+    return launch_reduce(out, partial_out, partial_lse, context_lens, B, Hq, D, partition_size, max_partitions, 0,
                          dtype, cs);
 }

@@ -31,7 +31,6 @@ namespace optgqa {
 
 namespace {
 
-constexpr int kD = 128;            // head dimension
 constexpr int kRows = 128;         // rows of the CTA's tiles (G heads x TQ tokens)
 constexpr int kTN = 64;            // keys per tile
 constexpr int kSub = 16;           // token rows per TMA box
@@ -42,31 +41,37 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: O is rescaled only when a row's maximum grew by more
 
 constexpr int kHalfBytes = kTN * 128;              // one 64-dim column half of a K or V tile (kTN rows of 128 B)
-constexpr int kTileBytes = 2 * kHalfBytes;         // a K or V tile
 constexpr int kQHalfBytes = kRows * 128;           // one 64-dim column half of the Q tile: 16 KiB
-constexpr int kQBytes = 2 * kQHalfBytes;
-constexpr int kOffQ = 0;
-constexpr int kOffK = kQBytes;
-constexpr int kOffV = kOffK + kKvStages * kTileBytes;
 // The ALiBi term rides on the tensor core as one more k-step of S = Q K^T: an extension of Q that holds
-// slope_h / scale split over three bf16 values, against an extension of K that holds the key's index inside
+// slope_h / |scale| split over three bf16 values, against an extension of K that holds the key's index inside
 // the tile three times.  Both are 16-dim K-major operands without swizzle: 8-row x 16-byte core matrices of
 // 128 contiguous bytes, the two 8-dim halves of a row group 128 bytes apart, row groups 256 bytes apart.
 constexpr int kExtRowGroupBytes = 256;
 constexpr int kQxBytes = kRows / 8 * kExtRowGroupBytes;   // 4 KiB
 constexpr int kKpBytes = kTN / 8 * kExtRowGroupBytes;     // 2 KiB
-constexpr int kOffQx = kOffV + kKvStages * kTileBytes;
-constexpr int kOffKp = kOffQx + kQxBytes;
-constexpr int kOffBar = kOffKp + kKpBytes;
-// barriers: q_full, k_full[3], k_empty[3], v_full[3], v_empty[3], s_full[2], p_full[2]; then the TMEM base word
+// barriers: q_full, k_full[], k_empty[], v_full[], v_empty[], s_full[2], p_full[2]; then the TMEM base word
 constexpr int kNumBars = 1 + 4 * kKvStages + 4;
-constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;   // + slack to align the tiles to 1 KiB
+
+// Shared memory of a CTA for head dimension D (64 or 128): the Q tile and the K/V rings as D / 64 column halves of
+// 128-byte rows, the extension operands, the barriers.
+template <int D>
+struct PfLayout {
+    static constexpr int kHalves = D / 64;
+    static constexpr int kTileBytes = kHalves * kHalfBytes;         // a K or V tile
+    static constexpr int kQBytes = kHalves * kQHalfBytes;
+    static constexpr int kOffQ = 0;
+    static constexpr int kOffK = kQBytes;
+    static constexpr int kOffV = kOffK + kKvStages * kTileBytes;
+    static constexpr int kOffQx = kOffV + kKvStages * kTileBytes;
+    static constexpr int kOffKp = kOffQx + kQxBytes;
+    static constexpr int kOffBar = kOffKp + kKpBytes;
+    static constexpr int kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;   // + slack to align the tiles to 1 KiB
+};
 
 // tensor-memory columns (fp32 accumulators, 128 lanes each)
 constexpr uint32_t kColS = 0;       // S buffers at 0 and kTN; P (bf16 pairs) overlays the first kTN / 2 columns of its S
-constexpr uint32_t kColO = 2 * kTN;
-constexpr uint32_t kTmemCols = kTN == 128 ? 512 : 256;    // a power of two >= 2 kTN + 128
-static_assert(kTN == 64 || kTN == 128, "tile of 64 or 128 keys");
+constexpr uint32_t kColO = 2 * kTN;                       // D columns
+constexpr uint32_t kTmemCols = 256;                       // a power of two >= 2 kTN + 128
 
 struct UmmaParams {
     __nv_bfloat16* out;
@@ -106,9 +111,11 @@ __device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr, uint32_t lbo_
            (1ull << 46);
 }
 
-// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128, N = n, A K-major, B K-major or MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major, uint32_t n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128, N = n, A K-major (optionally negated), B K-major
+// or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major, uint32_t n, bool negate_a = false) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((negate_a ? 1u : 0u) << 13) | ((b_mn_major ? 1u : 0u) << 16) |
+           ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // D[tmem] (+)= A[smem] * B[smem]
@@ -278,14 +285,17 @@ __device__ __forceinline__ float chunk_exp(const float (&v)[32], float qscale, f
 // kPaged: K/V come from the paged cache through block_tables (2-D maps over [rows, D]); otherwise from contiguous
 // k, v [tokens, Hkv, D] holding exactly the new tokens (3-D maps; the prompt branch with empty caches, where a
 // sequence's context is its own new tokens).
-template <int G, bool kPaged>
+template <int D, int G, bool kPaged>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const UmmaParams p) {
+    using L = PfLayout<D>;
+    constexpr int kTileBytes = L::kTileBytes, kOffQ = L::kOffQ, kOffK = L::kOffK, kOffV = L::kOffV, kOffQx = L::kOffQx,
+                  kOffKp = L::kOffKp;
     constexpr int TQ = kRows / G;     // new tokens per query block
     extern __shared__ char smem_raw[];
     char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kOffBar);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kOffBar);
     uint64_t* q_full = bars;
     uint64_t* k_full = bars + 1;
     uint64_t* k_empty = k_full + kKvStages;
@@ -333,13 +343,18 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tmem_slot[1] = 0;       // set by mbar_wait's callers when a wait gave up (see the end of the kernel)
         fence_barrier_init();
     }
-    // Extension operands of the ALiBi k-step (see kOffQx): row r of Q's holds slope_h / scale as a sum of three
-    // bf16 values, row e of K's the index e three times; dims 3..15 are zero.
-    const bool alibi = p.slopes != nullptr;
+    // The scale may have any sign.  The tensor core multiplies with |scale| in mind: a negative scale negates Q in
+    // the instruction (so that the row maximum can still be taken on the raw scores), a zero scale leaves the dot
+    // products out altogether and the scores are the bias alone.
+    const float sabs = p.scale == 0.f ? 1.f : fabsf(p.scale);
+    // Extension operands of the ALiBi k-step (see kOffQx): row r of Q's holds slope_h / |scale| as a sum of three
+    // bf16 values, row e of K's the index e three times; dims 3..15 are zero.  With a zero scale the step also
+    // runs without slopes (all-zero rows): it is then what initialises the score tile.
+    const bool alibi = p.slopes != nullptr || p.scale == 0.f;
     if (alibi) {
         if (threadIdx.x < kRows) {
             const int r = threadIdx.x;
-            const float a = p.slopes[kvh * G + r % G] / p.scale;
+            const float a = p.slopes ? p.slopes[kvh * G + r % G] / sabs : 0.f;
             const __nv_bfloat16 a0 = __float2bfloat16_rn(a);
             const __nv_bfloat16 a1 = __float2bfloat16_rn(a - __bfloat162float(a0));
             const __nv_bfloat16 a2 = __float2bfloat16_rn(a - __bfloat162float(a0) - __bfloat162float(a1));
@@ -372,9 +387,10 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (warp == 4) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            mbar_expect_tx(q_full, kQBytes);
-            tma_load_3d(smem + kOffQ, &map_q, 0, kvh * G, qstart + qb * TQ, q_full);
-            tma_load_3d(smem + kOffQ + kQHalfBytes, &map_q, 64, kvh * G, qstart + qb * TQ, q_full);
+            mbar_expect_tx(q_full, L::kQBytes);
+#pragma unroll
+            for (int hf = 0; hf < L::kHalves; ++hf)
+                tma_load_3d(smem + kOffQ + hf * kQHalfBytes, &map_q, 64 * hf, kvh * G, qstart + qb * TQ, q_full);
         }
         const int32_t* table = kPaged ? p.block_tables + (size_t)s * p.max_blocks : nullptr;
         const int sub = lane & 7;                           // lanes 0-7 fetch one 16-token slice each
@@ -393,30 +409,26 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             bool ok = true;
             if (j >= kKvStages) ok = mbar_wait(&k_empty[st], ((j / kKvStages) - 1) & 1, p.status);
             if (!__all_sync(kFull, ok)) break;
-            if (lane == 0) mbar_expect_tx(&k_full[st], (uint32_t)nsub * 2u * kSub * 128u);
+            if (lane == 0) mbar_expect_tx(&k_full[st], (uint32_t)nsub * L::kHalves * kSub * 128u);
             __syncwarp();
             if (lane < nsub) {
                 char* dst = smem + kOffK + st * kTileBytes + sub * (kSub * 128);
-                if (kPaged) {
-                    tma_load_2d(dst, &map_k, 0, row, &k_full[st]);
-                    tma_load_2d(dst + kHalfBytes, &map_k, 64, row, &k_full[st]);
-                } else {
-                    tma_load_3d(dst, &map_k, 0, kvh, qstart + tok, &k_full[st]);
-                    tma_load_3d(dst + kHalfBytes, &map_k, 64, kvh, qstart + tok, &k_full[st]);
+#pragma unroll
+                for (int hf = 0; hf < L::kHalves; ++hf) {
+                    if (kPaged) tma_load_2d(dst + hf * kHalfBytes, &map_k, 64 * hf, row, &k_full[st]);
+                    else tma_load_3d(dst + hf * kHalfBytes, &map_k, 64 * hf, kvh, qstart + tok, &k_full[st]);
                 }
             }
             if (j >= kKvStages) ok = mbar_wait(&v_empty[st], ((j / kKvStages) - 1) & 1, p.status);
             if (!__all_sync(kFull, ok)) break;
-            if (lane == 0) mbar_expect_tx(&v_full[st], (uint32_t)nsub * 2u * kSub * 128u);
+            if (lane == 0) mbar_expect_tx(&v_full[st], (uint32_t)nsub * L::kHalves * kSub * 128u);
             __syncwarp();
             if (lane < nsub) {
                 char* dst = smem + kOffV + st * kTileBytes + sub * (kSub * 128);
-                if (kPaged) {
-                    tma_load_2d(dst, &map_v, 0, row, &v_full[st]);
-                    tma_load_2d(dst + kHalfBytes, &map_v, 64, row, &v_full[st]);
-                } else {
-                    tma_load_3d(dst, &map_v, 0, kvh, qstart + tok, &v_full[st]);
-                    tma_load_3d(dst + kHalfBytes, &map_v, 64, kvh, qstart + tok, &v_full[st]);
+#pragma unroll
+                for (int hf = 0; hf < L::kHalves; ++hf) {
+                    if (kPaged) tma_load_2d(dst + hf * kHalfBytes, &map_v, 64 * hf, row, &v_full[st]);
+                    else tma_load_3d(dst + hf * kHalfBytes, &map_v, 64 * hf, kvh, qstart + tok, &v_full[st]);
                 }
             }
             page = page_next;
@@ -424,7 +436,9 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     } else if (warp == 5) {
         // ------------------------------------------------------------------ tensor-core issue (one thread)
         if (lane == 0) {
-            constexpr uint32_t idesc_s = instr_desc(false, kTN), idesc_pv = instr_desc(true, kD);
+            constexpr uint32_t idesc_s = instr_desc(false, kTN), idesc_pv = instr_desc(true, D);
+            const uint32_t idesc_qk = p.scale < 0.f ? instr_desc(false, kTN, true) : idesc_s;
+            const bool dots = p.scale != 0.f;
             const uint32_t q_addr = smem_u32(smem + kOffQ);
             bool ok = mbar_wait(q_full, 0, p.status);
             // O += P V for tile t: P (bf16 pairs, 8 columns per 16 keys) from tensor memory, V addressed MN-major:
@@ -449,15 +463,17 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 tc_fence_after();
                 // S = Q K^T: both K-major, 16 dims (32 bytes) per step inside the 128-byte swizzled rows
                 const uint32_t k_addr = smem_u32(smem + kOffK + st * kTileBytes);
+                if (dots) {
 #pragma unroll
-                for (int ks = 0; ks < kD / 16; ++ks) {
-                    umma_ss(tmem_base + kColS + sb * kTN,
-                            smem_desc(q_addr + (ks >> 2) * kQHalfBytes + (ks & 3) * 32, 16, 1024),
-                            smem_desc(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024), idesc_s, ks > 0);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        umma_ss(tmem_base + kColS + sb * kTN,
+                                smem_desc(q_addr + (ks >> 2) * kQHalfBytes + (ks & 3) * 32, 16, 1024),
+                                smem_desc(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024), idesc_qk, ks > 0);
+                    }
                 }
                 if (alibi)
                     umma_ss(tmem_base + kColS + sb * kTN, smem_desc_plain(smem_u32(smem + kOffQx), 128, kExtRowGroupBytes),
-                            smem_desc_plain(smem_u32(smem + kOffKp), 128, kExtRowGroupBytes), idesc_s, true);
+                            smem_desc_plain(smem_u32(smem + kOffKp), 128, kExtRowGroupBytes), idesc_s, dots);
                 tc_commit(&s_full[sb]);
                 tc_commit(&k_empty[st]);
                 if (j >= 1) ok = issue_pv(j - 1);
@@ -474,7 +490,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const int pos = n - qlen + min(i, i_last);
         const int lo = p.window > 0 ? pos - p.window : -1;       // keys lo < j <= pos are visible
         const int h = kvh * G + hg;
-        const float qscale = p.scale * kLog2e;
+        const float qscale = sabs * kLog2e;       // > 0: the tensor core has taken care of the scale's sign
         const float slope2 = p.slopes ? p.slopes[h] * kLog2e : 0.f;
         const float c_row = -slope2 * (float)pos;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
@@ -530,7 +546,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
-                for (int c = 0; c < kD / 32; ++c) {
+                for (int c = 0; c < D / 32; ++c) {
                     float v[32];
                     uint32_t w[32];
                     tmem_ld32(lane_addr + kColO + c * 32, v);
@@ -566,7 +582,7 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (r < kTN && j0 + r >= n) {
                     char* vrow = smem + kOffV + st * kTileBytes + r * 128;
 #pragma unroll
-                    for (int b = 0; b < 2; ++b)
+                    for (int b = 0; b < L::kHalves; ++b)
 #pragma unroll
                         for (int e = 0; e < 8; ++e)
                             *reinterpret_cast<uint4*>(vrow + b * kHalfBytes + e * 16) = make_uint4(0, 0, 0, 0);
@@ -585,9 +601,9 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (ok) {
             tc_fence_after();
             const float inv = 1.f / l;
-            uint4* orow = reinterpret_cast<uint4*>(p.out + ((size_t)(qstart + i) * p.Hq + h) * kD);
+            uint4* orow = reinterpret_cast<uint4*>(p.out + ((size_t)(qstart + i) * p.Hq + h) * D);
 #pragma unroll
-            for (int c = 0; c < kD / 32; ++c) {
+            for (int c = 0; c < D / 32; ++c) {
                 float v[32];
                 tmem_ld32(lane_addr + kColO + c * 32, v);
                 if (valid) {
@@ -618,59 +634,68 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
 }
 
-// q [tokens, Hq, 128] as a 3-D tensor; a box is 64 dims x the G heads of a group x 128 / G tokens, i.e. one
+// q [tokens, Hq, D] as a 3-D tensor; a box is 64 dims x the G heads of a group x 128 / G tokens, i.e. one
 // 64-dim half of the CTA's 128 rows, head-fastest.  Tokens past the end of q read as zeros.
-bool make_q_map(CUtensorMap* map, const void* q, int tokens, int Hq, int G) {
-    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hq, (cuuint64_t)tokens};
-    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hq * kD * 2};
+bool make_q_map(CUtensorMap* map, const void* q, int tokens, int Hq, int G, int D) {
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Hq, (cuuint64_t)tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hq * D * 2};
     const cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(kRows / G)};
     return make_bf16_map(map, q, 3, dims, strides, box);
 }
 
-// k or v [tokens, Hkv, 128] as a 3-D tensor; a box is 64 dims x one head x 16 tokens.
-bool make_kv_map(CUtensorMap* map, const void* kv, int tokens, int Hkv) {
-    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)Hkv, (cuuint64_t)tokens};
-    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)Hkv * kD * 2};
+// k or v [tokens, Hkv, D] as a 3-D tensor; a box is 64 dims x one head x 16 tokens.
+bool make_kv_map(CUtensorMap* map, const void* kv, int tokens, int Hkv, int D) {
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hkv * D * 2};
     const cuuint32_t box[3] = {64, 1, (cuuint32_t)kSub};
     return make_bf16_map(map, kv, 3, dims, strides, box);
 }
 
-template <int G, bool kPaged>
+template <int D, int G, bool kPaged>
 int launch_one(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& p, int B,
                int max_q_len, cudaStream_t stream) {
     static std::atomic<bool> configured[kMaxDevices];
-    if (!ensure_smem_limit(prefill_umma_kernel<G, kPaged>, kSmemBytes, configured)) return OPT_GQA_ERR_CUDA;
+    constexpr int kSmem = PfLayout<D>::kSmemBytes;
+    if (!ensure_smem_limit(prefill_umma_kernel<D, G, kPaged>, kSmem, configured)) return OPT_GQA_ERR_CUDA;
     constexpr int TQ = kRows / G;
     dim3 grid((max_q_len + TQ - 1) / TQ, p.Hkv, B);
-    return launch_dependent(prefill_umma_kernel<G, kPaged>, grid, dim3(kThreads), kSmemBytes, stream, mq, mk, mv, p);
+    return launch_dependent(prefill_umma_kernel<D, G, kPaged>, grid, dim3(kThreads), kSmem, stream, mq, mk, mv, p);
 }
 
-template <bool kPaged>
+template <int D, bool kPaged>
 int launch_g(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& p, int B, int G,
              int max_q_len, cudaStream_t stream) {
     switch (G) {
-        case 1: return launch_one<1, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
-        case 2: return launch_one<2, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
-        case 4: return launch_one<4, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
-        case 8: return launch_one<8, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+        case 1: return launch_one<D, 1, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+        case 2: return launch_one<D, 2, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+        case 4: return launch_one<D, 4, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
+        case 8: return launch_one<D, 8, kPaged>(mq, mk, mv, p, B, max_q_len, stream);
     }
+    return OPT_GQA_ERR_SHAPE;
+}
+
+template <bool kPaged>
+int launch_d(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const UmmaParams& p, int B, int G,
+             int D, int max_q_len, cudaStream_t stream) {
+    if (D == 128) return launch_g<128, kPaged>(mq, mk, mv, p, B, G, max_q_len, stream);
+    if (D == 64) return launch_g<64, kPaged>(mq, mk, mv, p, B, G, max_q_len, stream);
     return OPT_GQA_ERR_SHAPE;
 }
 
 }  // namespace
 
-// bf16, D = 128 only.
+// bf16, D = 64 or 128, any scale; window > 0 adds the local mask.
 int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, int total_q_tokens, int max_q_len,
                         const void* k_cache, const void* v_cache, const int32_t* block_tables, int max_blocks_per_seq,
                         const int32_t* context_lens, const float* alibi_slopes, float scale, int B, int Hq, int Hkv,
-                        int bs, int64_t num_blocks, int window, int* device_status, cudaStream_t stream) {
+                        int D, int bs, int64_t num_blocks, int window, int* device_status, cudaStream_t stream) {
     const uint64_t rows = (uint64_t)num_blocks * (uint64_t)Hkv * (uint64_t)bs;
     if (rows == 0 || rows > 0x7fffffffull || total_q_tokens <= 0) return OPT_GQA_ERR_SHAPE;
     if (B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
     const int G = Hq / Hkv;
     CUtensorMap mq, mk, mv;
-    if (!make_q_map(&mq, q, total_q_tokens, Hq, G) || !make_cache_map(&mk, k_cache, rows, kD, kSub) ||
-        !make_cache_map(&mv, v_cache, rows, kD, kSub))
+    if (!make_q_map(&mq, q, total_q_tokens, Hq, G, D) || !make_cache_map(&mk, k_cache, rows, D, kSub) ||
+        !make_cache_map(&mv, v_cache, rows, D, kSub))
         return OPT_GQA_ERR_CUDA;
     UmmaParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
@@ -685,18 +710,18 @@ int launch_prefill_umma(void* out, const void* q, const int32_t* q_start_loc, in
     p.Hkv = Hkv;
     p.bs = bs;
     p.window = window;
-    return launch_g<true>(mq, mk, mv, p, B, G, max_q_len, stream);
+    return launch_d<true>(mq, mk, mv, p, B, G, D, max_q_len, stream);
 }
 
-// The prompt branch with empty caches: q [tokens, Hq, 128], k, v [tokens, Hkv, 128] contiguous, causal + ALiBi.
+// The prompt branch with empty caches: q [tokens, Hq, D], k, v [tokens, Hkv, D] contiguous, causal + ALiBi.
 int launch_prompt_umma(void* out, const void* q, const void* k, const void* v, const int32_t* q_start_loc,
                        int total_q_tokens, int max_q_len, const float* alibi_slopes, float scale, int B, int Hq,
-                       int Hkv, int* device_status, cudaStream_t stream) {
+                       int Hkv, int D, int* device_status, cudaStream_t stream) {
     if (total_q_tokens <= 0 || B > 65535 || Hkv > 65535) return OPT_GQA_ERR_SHAPE;
     const int G = Hq / Hkv;
     CUtensorMap mq, mk, mv;
-    if (!make_q_map(&mq, q, total_q_tokens, Hq, G) || !make_kv_map(&mk, k, total_q_tokens, Hkv) ||
-        !make_kv_map(&mv, v, total_q_tokens, Hkv))
+    if (!make_q_map(&mq, q, total_q_tokens, Hq, G, D) || !make_kv_map(&mk, k, total_q_tokens, Hkv, D) ||
+        !make_kv_map(&mv, v, total_q_tokens, Hkv, D))
         return OPT_GQA_ERR_CUDA;
     UmmaParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
@@ -711,7 +736,7 @@ int launch_prompt_umma(void* out, const void* q, const void* k, const void* v, c
     p.Hkv = Hkv;
     p.bs = 16;
     p.window = 0;
-    return launch_g<false>(mq, mk, mv, p, B, G, max_q_len, stream);
+    return launch_d<false>(mq, mk, mv, p, B, G, D, max_q_len, stream);
 }
 
 }  // namespace optgqa

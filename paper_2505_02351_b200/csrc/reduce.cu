@@ -19,7 +19,7 @@ constexpr int kReducePre = 8;
 template <typename T, int D>
 __global__ void __launch_bounds__(kReduceWarps * 32)
 reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const float* __restrict__ partial_lse,
-              const int32_t* __restrict__ context_lens, int Hq, int partition_size, int max_partitions) {
+              const int32_t* __restrict__ context_lens, int Hq, int partition_size, int max_partitions, int window) {
     constexpr int V = D / 32;             // columns per lane
     using Vec = typename std::conditional<V == 4, float4, float2>::type;
     __shared__ float s_num[kReduceWarps][D];
@@ -32,9 +32,11 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
     // never beyond the rows the decode grid had (max_partitions is the caller's promise; a length that breaks it gives
     // a wrong row, not a read past the partials)
     const int np = min((n + partition_size - 1) / partition_size, max_partitions);
+    // with a local mask the partitions wholly before the first attended key hold nothing
+    const int p_lo = window > 0 ? max(0, n - window) / partition_size : 0;
     T* o = out + (size_t)row * D;
     grid_dependency_wait();                // the partials come from the decode grid; out may still be read by its last user
-    if (np <= 0) {
+    if (np <= p_lo) {
         for (int d = threadIdx.x; d < D; d += blockDim.x) o[d] = T(0.f);
         return;
     }
@@ -45,7 +47,7 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
     Vec xpre[kReducePre];
 #pragma unroll
     for (int k = 0; k < kReducePre; ++k) {
-        const int p = warp + k * kReduceWarps;
+        const int p = p_lo + warp + k * kReduceWarps;
         lpre[k] = -INFINITY;
         if (p < np) {
             lpre[k] = lse[p];
@@ -53,7 +55,7 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
         }
     }
     float L = -INFINITY;
-    for (int p = lane; p < np; p += 32) L = fmaxf(L, lse[p]);
+    for (int p = p_lo + lane; p < np; p += 32) L = fmaxf(L, lse[p]);
 #pragma unroll
     for (int o2 = 16; o2 >= 1; o2 >>= 1) L = fmaxf(L, __shfl_xor_sync(0xffffffffu, L, o2));
 
@@ -73,9 +75,9 @@ reduce_kernel(T* __restrict__ out, const float* __restrict__ partial_out, const 
     };
 #pragma unroll
     for (int k = 0; k < kReducePre; ++k)
-        if (warp + k * kReduceWarps < np) add_row(lpre[k], xpre[k]);
+        if (p_lo + warp + k * kReduceWarps < np) add_row(lpre[k], xpre[k]);
 #pragma unroll 4
-    for (int p = warp + kReducePre * kReduceWarps; p < np; p += kReduceWarps)
+    for (int p = p_lo + warp + kReducePre * kReduceWarps; p < np; p += kReduceWarps)
         add_row(lse[p], *reinterpret_cast<const Vec*>(po + (size_t)p * D));
 #pragma unroll
     for (int v = 0; v < V; ++v) s_num[warp][lane * V + v] = num[v];
@@ -238,26 +240,27 @@ reduce_balanced_kernel(T* __restrict__ out, const float* __restrict__ partial_ou
 template <typename T, int D>
 static int launch_reduce_t(void* out, const float* partial_out, const float* partial_lse,
                            const int32_t* context_lens, int B, int Hq, int partition_size, int max_partitions,
-                           cudaStream_t stream) {
+                           int window, cudaStream_t stream) {
     return launch_dependent(reduce_kernel<T, D>, dim3((unsigned)B * (unsigned)Hq), dim3(kReduceWarps * 32), 0, stream,
                             static_cast<T*>(out), partial_out, partial_lse, context_lens, Hq, partition_size,
-                            max_partitions);
+                            max_partitions, window);
 }
 
 int launch_reduce(void* out, const float* partial_out, const float* partial_lse, const int32_t* context_lens,
-                  int B, int Hq, int D, int partition_size, int max_partitions, int dtype, cudaStream_t stream) {
+                  int B, int Hq, int D, int partition_size, int max_partitions, int window, int dtype,
+                  cudaStream_t stream) {
     if (dtype == OPT_GQA_BF16) {
         if (D == 128)
             return launch_reduce_t<__nv_bfloat16, 128>(out, partial_out, partial_lse, context_lens, B, Hq,
-                                                       partition_size, max_partitions, stream);
+                                                       partition_size, max_partitions, window, stream);
         return launch_reduce_t<__nv_bfloat16, 64>(out, partial_out, partial_lse, context_lens, B, Hq, partition_size,
-                                                  max_partitions, stream);
+                                                  max_partitions, window, stream);
     }
     if (D == 128)
         return launch_reduce_t<float, 128>(out, partial_out, partial_lse, context_lens, B, Hq, partition_size,
-                                           max_partitions, stream);
+                                           max_partitions, window, stream);
     return launch_reduce_t<float, 64>(out, partial_out, partial_lse, context_lens, B, Hq, partition_size,
-                                      max_partitions, stream);
+                                      max_partitions, window, stream);
 }
 
 template <typename T, int D, int WPR, int kPre = 0>

@@ -71,17 +71,56 @@ def test_prefill_local_window(window, Hq, Hkv):
         assert np.max(np.abs(got - _oracle(wl, window, slopes))) <= TOL, (window, slopes)
 
 
+@pytest.mark.parametrize("window", [1, 16, 17, 100, 5000])
+@pytest.mark.parametrize("D", [64, 128])
+def test_decode_local_window_on_fp32_caches(window, D):
+    """fp32 caches: one partial per partition on the CUDA-core kernel, merge over the partitions inside the window."""
+    wl = W.make_custom("win32", "fp32", 8, 2, D, 16, [1, 15, 16, 17, 33, 100, 257, 0, 640], seed=83, poison=True)
+    d = util.DeviceWorkload(wl)
+    binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
+    for P in (32, 512):
+        maxP = (int(wl.context_lens.max()) + P - 1) // P
+        ws = torch.full((wl.B * wl.Hq * maxP * (wl.D + 1),), float("nan"), device="cuda:0")
+        for slopes in (False, True):
+            d.out.fill_(float("nan"))
+            binding.paged_attention_decode_local(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+                                                 d.alibi_slopes if slopes else None, wl.scale, P, ws, maxP, window)
+            torch.cuda.synchronize()
+            assert binding.device_status() == 0
+            got = d.out.double().cpu().numpy()
+            assert np.isfinite(got).all()
+            assert np.max(np.abs(got - _oracle(wl, window, slopes))) <= util.TOL["fp32"], (window, P, slopes)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("scale", [0.0, -0.07, 0.2])
+def test_prefill_local_window_head_dims_and_scales(D, scale):
+    """The windowed chunked prefill on tcgen05 for head dimension 64 and for scales that are zero or negative."""
+    lens = [700, 77, 130, 1, 300]
+    qls = [300, 77, 129, 1, 17]
+    wl = W.make_custom("winpf2", "bf16", 8, 2, D, 32, lens, q_lens=qls, seed=84, poison=True, scale=scale)
+    d = util.DeviceWorkload(wl)
+    binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
+    for window, slopes in ((40, True), (200, False), (64, True)):
+        d.out.fill_(float("nan"))
+        binding.paged_attention_prefill_local(d.out, d.q, d.q_start_loc, max(qls), d.k_cache, d.v_cache, d.block_tables,
+                                              d.context_lens, d.alibi_slopes if slopes else None, wl.scale, window)
+        torch.cuda.synchronize()
+        assert binding.device_status() == 0
+        got = d.out.double().cpu().numpy()
+        assert np.isfinite(got).all()
+        assert np.max(np.abs(got - _oracle(wl, window, slopes))) <= TOL, (window, slopes)
+
+
 def test_window_entry_points_reject_what_they_do_not_support():
-    wl = W.make_config(1)      # fp32
+    wl = W.make_custom("w0", "bf16", 8, 2, 128, 16, [64], seed=82)
     d = util.DeviceWorkload(wl)
     ws = torch.empty(binding.workspace_bytes(wl.B, wl.Hq, wl.D, 8), dtype=torch.uint8, device="cuda:0")
     with pytest.raises(binding.OptGqaError) as e:
         binding.paged_attention_decode_local(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, None,
-                                             wl.scale, 16, ws, 8, 4)
-    assert e.value.code == -3          # fp32 caches
-    wl = W.make_custom("w0", "bf16", 8, 2, 128, 16, [64], seed=82)
-    d = util.DeviceWorkload(wl)
-    with pytest.raises(binding.OptGqaError) as e:
-        binding.paged_attention_decode_local(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens, None,
                                              wl.scale, 16, ws, 8, 0)
     assert e.value.code == -2          # window must be positive
+    with pytest.raises(binding.OptGqaError) as e:
+        binding.paged_attention_prefill_local(d.out, d.q, torch.zeros(2, dtype=torch.int32, device="cuda:0"), 1,
+                                              d.k_cache, d.v_cache, d.block_tables, d.context_lens, None, wl.scale, 0)
+    assert e.value.code == -2

@@ -28,10 +28,9 @@ def test_shape_matrix_ragged_chunks(D, Hq, Hkv, bs):
     lens = [200, 77, 33, 130, 1, 64, 300]
     qls = [70, 77, 1, 129, 1, 16, 17]
     wl = W.make_custom("pf", "bf16", Hq, Hkv, D, bs, lens, q_lens=qls, seed=D + Hq + bs, poison=True)
-    _check(wl)
+    _check(wl)                   # the default entry point runs on tcgen05 for both head dimensions
     _check(wl, slopes=False)
-    if D == 128:                 # the default entry point ran on tcgen05: also the warp-level kernel
-        _check(wl, mma=True)
+    _check(wl, mma=True)         # the warp-level kernel
 
 
 def test_tiles_and_blocks_boundaries_on_tcgen05():
@@ -73,11 +72,15 @@ def test_prefill_with_one_new_token_is_the_decode_result():
 
 @pytest.mark.parametrize("scale", [0.0, -0.05, 0.5])
 def test_scales_that_are_not_the_usual_one(scale):
-    """The tcgen05 kernel needs a positive scale (it takes the row maximum before scaling); zero and negative
-    scales are routed to the other kernel.  Either way the result is the oracle's."""
-    wl = W.make_custom("pfs", "bf16", 8, 2, 128, 16, [300, 70], q_lens=[130, 70], seed=37)
-    wl.scale = scale
-    _check(wl)
+    """The tcgen05 kernel takes the row maximum on the raw scores, which needs a positive factor: a negative scale
+    negates Q inside the tensor-core instruction, a zero scale leaves the dot products out.  Both kernels, both head
+    dimensions: the result is the oracle's."""
+    for D in (128, 64):
+        wl = W.make_custom("pfs", "bf16", 8, 2, D, 16, [300, 70], q_lens=[130, 70], seed=37)
+        wl.scale = scale
+        _check(wl)
+        _check(wl, slopes=False)
+        _check(wl, mma=True)
 
 
 def test_steep_and_flat_slopes_on_the_tensor_core_bias():
@@ -156,10 +159,19 @@ def test_prompt_attention_equals_prefill_over_the_appended_cache():
     assert np.array_equal(got, paged)         # same kernel, same tiles, same order: bitwise equal
 
 
+@pytest.mark.parametrize("scale", [None, 0.0, -0.1])
+def test_prompt_attention_head_dim_64_and_other_scales(scale):
+    for D in (64, 128):
+        lens = [200, 77, 1, 129, 64]
+        wl = W.make_custom("prompt3", "bf16", 8, 2, D, 16, lens, q_lens=lens, seed=76, scale=scale)
+        _prompt(wl)
+        _prompt(wl, slopes=False)
+
+
 def test_prompt_attention_rejects_what_it_does_not_support():
-    wl = W.make_custom("prompt3", "bf16", 4, 2, 64, 16, [10], q_lens=[10], seed=76)
+    wl = W.make_custom("prompt4", "bf16", 4, 2, 64, 16, [10], q_lens=[10], seed=77)
     q = wl.q.cuda()
     with pytest.raises(binding.OptGqaError) as e:
-        binding.prompt_attention(torch.empty_like(q), q, wl.k_new.cuda(), wl.v_new.cuda(), wl.q_start_loc.cuda(), 10,
-                                 None, wl.scale)
-    assert e.value.code == -2                 # head_dim 64 is not built for this entry point
+        binding.prompt_attention(torch.empty_like(q), q.float(), wl.k_new.cuda().float(), wl.v_new.cuda().float(),
+                                 wl.q_start_loc.cuda(), 10, None, wl.scale)
+    assert e.value.code == -3                 # fp32 tensors: the entry point is bf16 only
