@@ -563,15 +563,29 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // (a row that has not seen a key yet has only -inf scores: subtract 0 so that they give p = 0)
             const float m_sub = m_used == -INFINITY ? 0.f : m_used;
             const float bias_m = bias0 - m_sub;
-            float sum = 0.f;
-#pragma unroll
-            for (int c = 0; c < kTN / 32; ++c) {
+            // Far from the diagonal the ALiBi term alone puts every score of the tile more than 127 binary orders
+            // below the row's reference maximum: 2^(s - m) is then exactly zero in this arithmetic (the exponential
+            // flushes results below 2^-126 to zero), for every key of the tile.  Where that holds for all rows of
+            // the warp, the exponentials are not evaluated: P is written as zeros, the denominator stays as it is.
+            // (The tensor core still multiplies the tile: nothing is skipped there.)
+            const bool all_zero = __all_sync(kFull, m_tile - m_used < -127.f);
+            if (all_zero) {
                 uint32_t w[16];
-                if (masked) sum += chunk_exp<true>(v[c], qscale, bias_m, j0 + c * 32, pos, lo, w);
-                else sum += chunk_exp<false>(v[c], qscale, bias_m, j0 + c * 32, pos, lo, w);
-                tmem_st16(s_addr + c * 16, w);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) w[e] = 0u;
+#pragma unroll
+                for (int c = 0; c < kTN / 32; ++c) tmem_st16(s_addr + c * 16, w);
+            } else {
+                float sum = 0.f;
+#pragma unroll
+                for (int c = 0; c < kTN / 32; ++c) {
+                    uint32_t w[16];
+                    if (masked) sum += chunk_exp<true>(v[c], qscale, bias_m, j0 + c * 32, pos, lo, w);
+                    else sum += chunk_exp<false>(v[c], qscale, bias_m, j0 + c * 32, pos, lo, w);
+                    tmem_st16(s_addr + c * 16, w);
+                }
+                l += sum;
             }
-            l += sum;
 
             if (j0 + kTN > n) {
                 // Rows past the end of the sequence hold whatever the page held, or stale shared memory where no
