@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 DEFAULT_PARTITION = {2: 256, 3: 512, 4: 512}
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised
 # under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {3: 378_693_376 + 3_752_704}   # profiles/decode_stream_cfg3.md
+NCU_TRAFFIC_BYTES = {3: 378_703_104 + 3_860_992}   # profiles/decode_stream_cfg3.md
 KERNEL_TIMING_STEPS = 512   # steps of the kernel-timing region (a bracket every EVENT_EVERY-th step)
 E2E_STEPS = 200             # steps of the end-to-end leg
 READ_PROBE_BYTES = 1 << 30  # bytes streamed by the read-only ceiling probe per launch
@@ -598,7 +598,8 @@ def read_only_ceiling(dev, stream) -> dict:
 
 
 def run_e2e(batch: DeviceBatch, steps: int, warmup: int):
-    """Steps through opt_gqa_decode_step_host: pinned host inputs copied in, result copied out, every step."""
+    """Steps through opt_gqa_decode_step_mapped: pinned host inputs brought in, result stored back, every step (the
+    buffers' device-side addresses are those torch's pinned allocations have under unified addressing)."""
     import torch
 
     from paper_2505_02351_b200 import binding
@@ -623,7 +624,7 @@ def run_e2e(batch: DeviceBatch, steps: int, warmup: int):
                batch.ws_bytes if batch.P else 0, batch.maxP, batch.dt, sh) for i in range(R)]
 
     def step(i):
-        check(lib.opt_gqa_decode_step_host(*a_host[i % R]), "decode_step_host")
+        check(lib.opt_gqa_decode_step_mapped(*a_host[i % R]), "decode_step_mapped")
         stream.synchronize()          # the caller reads out_host after every step
 
     for i in range(warmup):
@@ -807,7 +808,7 @@ def main():
         e2e_s = max_over_ranks(e2e_s, str(dev))
         e2e = {"value": tokens_all * E2E_STEPS / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": E2E_STEPS, "us_per_step": e2e_s / E2E_STEPS * 1e6,
-               "api": "opt_gqa_decode_step_host (pinned host q/k_new/v_new/slots/tables/lens in, out back, "
+               "api": "opt_gqa_decode_step_mapped (pinned host q/k_new/v_new/slots/tables/lens in, out back, "
                       "stream synchronised per step)"}
         e2e["frac_of_value"] = e2e["value"] / value
         ceiling = read_only_ceiling(dev, torch.cuda.current_stream())

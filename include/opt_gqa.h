@@ -381,6 +381,21 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
                              int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
                              size_t workspace_bytes, int max_partitions, int dtype, void* stream);
 
+/*
+ * opt_gqa_decode_step_host for a caller that has looked the device-side addresses of its page-locked
+ * buffers up once (cudaHostGetDevicePointer; with unified addressing, memory from cudaHostAlloc /
+ * cudaMallocHost has the same address on both sides): the seven *_view arguments are those addresses,
+ * the call makes no pointer queries, and the transfers are always done by the kernels themselves (one
+ * gather kernel in, out stored by the step's last kernel).  Views must be 4-byte aligned, out_view
+ * 16-byte aligned (OPT_GQA_ERR_ALIGN otherwise).  Everything else as in opt_gqa_decode_step_host.
+ */
+int opt_gqa_decode_step_mapped(void* out_view, const void* q_view, const void* k_new_view, const void* v_new_view,
+                               const int64_t* slot_mapping_view, const int32_t* block_tables_view,
+                               const int32_t* context_lens_view, void* staging, void* k_cache, void* v_cache,
+                               int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
+                               int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
+                               size_t workspace_bytes, int max_partitions, int dtype, void* stream);
+
 /* Device bytes opt_gqa_decode_step_host needs in `staging`.  Host arithmetic; 0 for bad arguments. */
 size_t opt_gqa_step_staging_bytes(int B, int Hq, int Hkv, int D, int max_blocks_per_seq, int dtype);
 

@@ -51,6 +51,8 @@ SIGNATURES = {
                                  _i, _vp, _sz, _i, _i, _vp]),
     "opt_gqa_decode_step_host": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _f, _i, _i, _i, _i,
                                       _i, _i64, _i, _vp, _sz, _i, _i, _vp]),
+    "opt_gqa_decode_step_mapped": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _f, _i, _i, _i, _i,
+                                        _i, _i64, _i, _vp, _sz, _i, _i, _vp]),
     "opt_gqa_step_staging_bytes": (_c.c_size_t, [_i, _i, _i, _i, _i, _i]),
     "opt_gqa_workspace_bytes": (_c.c_size_t, [_i, _i, _i, _i]),
     "opt_gqa_debug_wait_timeout": (_i, [_c.c_longlong, _vp]),
@@ -323,3 +325,25 @@ def decode_step_host(out_host, q_host, k_new_host, v_new_host, slot_mapping_host
         _ptr(k_cache), _ptr(v_cache), block_tables_host.shape[1], _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs,
         num_blocks, partition_size, _ptr(workspace), _nbytes(workspace), max_partitions, _DTYPE_CODE[q_host.dtype],
         _stream(stream)), "opt_gqa_decode_step_host")
+
+
+def _pinned_view(t: torch.Tensor) -> int:
+    """Device-side address of a page-locked host tensor.  torch allocates pinned memory with cudaHostAlloc, whose
+    device-side address under unified addressing is the host address itself."""
+    if t.is_cuda or not t.is_contiguous() or not t.is_pinned():
+        raise ValueError("expected a contiguous page-locked (pinned) host tensor")
+    return t.data_ptr()
+
+
+def decode_step_mapped(out_host, q_host, k_new_host, v_new_host, slot_mapping_host, block_tables_host,
+                       context_lens_host, staging, k_cache, v_cache, alibi_slopes, scale: float,
+                       partition_size: int = 0, workspace=None, max_partitions: int = 0, stream=None) -> None:
+    """decode_step_host for pinned tensors whose device-side addresses are passed as they are (no pointer queries)."""
+    B, Hq, D = q_host.shape
+    num_blocks, Hkv, bs, _ = k_cache.shape
+    _check(load().opt_gqa_decode_step_mapped(
+        _pinned_view(out_host), _pinned_view(q_host), _pinned_view(k_new_host), _pinned_view(v_new_host),
+        _pinned_view(slot_mapping_host), _pinned_view(block_tables_host), _pinned_view(context_lens_host), _ptr(staging),
+        _ptr(k_cache), _ptr(v_cache), block_tables_host.shape[1], _ptr(alibi_slopes), scale, B, Hq, Hkv, D, bs,
+        num_blocks, partition_size, _ptr(workspace), _nbytes(workspace), max_partitions, _DTYPE_CODE[q_host.dtype],
+        _stream(stream)), "opt_gqa_decode_step_mapped")

@@ -453,12 +453,16 @@ size_t opt_gqa_step_staging_bytes(int B, int Hq, int Hkv, int D, int max_blocks_
     return staging_layout(B, Hq, Hkv, D, max_blocks_per_seq, dtype, &L) ? L.total : 0;
 }
 
-int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_new_host, const void* v_new_host,
-                             const int64_t* slot_mapping_host, const int32_t* block_tables_host,
-                             const int32_t* context_lens_host, void* staging, void* k_cache, void* v_cache,
-                             int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
-                             int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
-                             size_t workspace_bytes, int max_partitions, int dtype, void* stream) {
+extern "C++" {
+// The step from host buffers.  kResolved: the seven pointers are already the device-side addresses of page-locked
+// memory (the caller looked them up once), so the per-call pointer queries are left out.
+template <bool kResolved>
+static int host_step(void* out_host, const void* q_host, const void* k_new_host, const void* v_new_host,
+                     const int64_t* slot_mapping_host, const int32_t* block_tables_host,
+                     const int32_t* context_lens_host, void* staging, void* k_cache, void* v_cache,
+                     int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq, int Hkv, int D,
+                     int bs, int64_t num_blocks, int partition_size, void* workspace, size_t workspace_bytes,
+                     int max_partitions, int dtype, void* stream) {
     if (!dtype_ok(dtype)) return OPT_GQA_ERR_DTYPE;
     if (B < 0 || !shape_ok(Hq, Hkv, D, bs) || max_blocks_per_seq < 0) return OPT_GQA_ERR_SHAPE;
     if (B == 0) return OPT_GQA_OK;
@@ -487,8 +491,8 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
     HostGather g;
     bool pinned = true, wide = true;
     for (int a = 0; a < 6; ++a) {
-        const void* dv = device_view(src[a]);
-        pinned &= dv != nullptr && bytes[a] % 4 == 0;
+        const void* dv = kResolved ? src[a] : device_view(src[a]);
+        pinned &= dv != nullptr && bytes[a] % 4 == 0 && (reinterpret_cast<uintptr_t>(dv) & 3u) == 0;
         wide &= bytes[a] % 16 == 0 && (reinterpret_cast<uintptr_t>(dv) & 15u) == 0;
         g.src[a] = dv;
         g.dst[a] = st + off[a];
@@ -501,8 +505,9 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
     }
     pinned &= words <= 0x7fffffffull;
     g.first[6] = (unsigned)words;
-    void* out_dev = pinned ? const_cast<void*>(device_view(out_host)) : nullptr;
+    void* out_dev = !pinned ? nullptr : kResolved ? out_host : const_cast<void*>(device_view(out_host));
     pinned &= out_dev != nullptr && (reinterpret_cast<uintptr_t>(out_dev) & 15u) == 0;
+    if (kResolved && !pinned) return OPT_GQA_ERR_ALIGN;     // views must be 4-byte aligned, the one of out 16-byte
     if (pinned) {
         const unsigned ctas = (unsigned)((words + 255) / 256 < 148 ? (words + 255) / 256 : 148);
         if (wide) gather_host_kernel<uint4><<<ctas, 256, 0, cs>>>(g);
@@ -524,6 +529,31 @@ int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_n
     if (!pinned && cudaMemcpyAsync(out_host, st + L.out, qb, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
         return OPT_GQA_ERR_CUDA;
     return OPT_GQA_OK;
+}
+}  // extern "C++"
+
+int opt_gqa_decode_step_host(void* out_host, const void* q_host, const void* k_new_host, const void* v_new_host,
+                             const int64_t* slot_mapping_host, const int32_t* block_tables_host,
+                             const int32_t* context_lens_host, void* staging, void* k_cache, void* v_cache,
+                             int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
+                             int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
+                             size_t workspace_bytes, int max_partitions, int dtype, void* stream) {
+    return host_step<false>(out_host, q_host, k_new_host, v_new_host, slot_mapping_host, block_tables_host,
+                            context_lens_host, staging, k_cache, v_cache, max_blocks_per_seq, alibi_slopes, scale, B, Hq,
+                            Hkv, D, bs, num_blocks, partition_size, workspace, workspace_bytes, max_partitions, dtype,
+                            stream);
+}
+
+int opt_gqa_decode_step_mapped(void* out_view, const void* q_view, const void* k_new_view, const void* v_new_view,
+                               const int64_t* slot_mapping_view, const int32_t* block_tables_view,
+                               const int32_t* context_lens_view, void* staging, void* k_cache, void* v_cache,
+                               int max_blocks_per_seq, const float* alibi_slopes, float scale, int B, int Hq,
+                               int Hkv, int D, int bs, int64_t num_blocks, int partition_size, void* workspace,
+                               size_t workspace_bytes, int max_partitions, int dtype, void* stream) {
+    return host_step<true>(out_view, q_view, k_new_view, v_new_view, slot_mapping_view, block_tables_view,
+                           context_lens_view, staging, k_cache, v_cache, max_blocks_per_seq, alibi_slopes, scale, B, Hq,
+                           Hkv, D, bs, num_blocks, partition_size, workspace, workspace_bytes, max_partitions, dtype,
+                           stream);
 }
 
 size_t opt_gqa_workspace_bytes(int B, int Hq, int D, int max_partitions) {

@@ -253,9 +253,10 @@ def test_largest_group_and_smallest_head_dim():
     _check(wl32, partition_size=128)
 
 
-@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("pinned", [True, False, "mapped"])
 def test_decode_step_from_host_buffers(pinned):
-    """opt_gqa_decode_step_host: pinned buffers are read and written by the kernels directly, pageable ones are copied."""
+    """opt_gqa_decode_step_host: pinned buffers are read and written by the kernels directly, pageable ones are copied;
+    opt_gqa_decode_step_mapped takes the pinned buffers' device-side addresses without looking them up."""
     for wl, P in ((W.make_config(3, shrink=8), 512), (W.make_config(1), 0)):
         d = util.DeviceWorkload(wl)
         pin = (lambda t: t.contiguous().pin_memory()) if pinned else (lambda t: t.contiguous().clone())
@@ -267,8 +268,9 @@ def test_decode_step_from_host_buffers(pinned):
         staging = torch.empty(binding.step_staging_bytes(wl.B, wl.Hq, wl.Hkv, wl.D, wl.max_blocks, tdt), dtype=torch.uint8,
                               device="cuda:0")
         ws = torch.empty(max(16, binding.workspace_bytes(wl.B, wl.Hq, wl.D, maxP)), dtype=torch.uint8, device="cuda:0")
-        binding.decode_step_host(hout, hq, hk, hv, hs, ht, hl, staging, d.k_cache, d.v_cache, d.alibi_slopes, wl.scale,
-                                 partition_size=P, workspace=ws if P else None, max_partitions=maxP)
+        step = binding.decode_step_mapped if pinned == "mapped" else binding.decode_step_host
+        step(hout, hq, hk, hv, hs, ht, hl, staging, d.k_cache, d.v_cache, d.alibi_slopes, wl.scale,
+             partition_size=P, workspace=ws if P else None, max_partitions=maxP)
         torch.cuda.synchronize()
         assert binding.device_status() == 0
         want = util.oracle_attention(wl)
