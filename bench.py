@@ -336,7 +336,8 @@ def prefill_report(dev, steps: int, warmup: int) -> dict:
             "launches_timed": steps, "flop_per_launch": pb.flops(), "bound": "tensor"}
 
 
-PROJECTION_SHAPES = (("width4096_32q4kv_T8", 8, 4096, 32, 4, 128), ("width8192_64q8kv_T8", 8, 8192, 64, 8, 128),
+# the 70B-like shape first: a profiler capture of the first launches (--only projection) lands on it
+PROJECTION_SHAPES = (("width8192_64q8kv_T8", 8, 8192, 64, 8, 128), ("width4096_32q4kv_T8", 8, 4096, 32, 4, 128),
                      ("width8192_64q8kv_T16", 16, 8192, 64, 8, 128))
 
 
