@@ -34,7 +34,7 @@ namespace {
 constexpr int kRows = 128;         // rows of the CTA's tiles (G heads x TQ tokens)
 constexpr int kTN = 64;            // keys per tile
 constexpr int kSub = 16;           // token rows per TMA box
-constexpr int kKvStages = 2;
+constexpr int kKvStages = 2;       // (the issuing thread selects a stage's descriptors with one compare: two stages)
 constexpr int kCtasPerSm = 2;
 constexpr int kThreads = 192;
 constexpr unsigned kFull = 0xffffffffu;
@@ -109,6 +109,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 __device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
            (1ull << 46);
+}
+
+// The descriptor of the same layout `bytes` further on in shared memory (a multiple of 16; the address field counts
+// 16-byte units and shared memory ends below 2^18, so only the low word changes): one add where building a
+// descriptor anew costs several instructions of the one thread that issues all tensor-core work.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) {
+    return (desc & 0xFFFFFFFF00000000ull) | (uint32_t)((uint32_t)desc + (bytes >> 4));
 }
 
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128, N = n, A K-major (optionally negated), B K-major
@@ -439,7 +446,19 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             constexpr uint32_t idesc_s = instr_desc(false, kTN), idesc_pv = instr_desc(true, D);
             const uint32_t idesc_qk = p.scale < 0.f ? instr_desc(false, kTN, true) : idesc_s;
             const bool dots = p.scale != 0.f;
-            const uint32_t q_addr = smem_u32(smem + kOffQ);
+            // Every descriptor that does not change from tile to tile is built once: Q's for the D / 16 k-steps, the
+            // extension operands', and per ring stage those of the K tile's first k-step and the V tile's first 16 keys.
+            uint64_t q_desc[D / 16], k_desc0[kKvStages], v_desc0[kKvStages];
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+                q_desc[ks] = smem_desc(smem_u32(smem + kOffQ) + (ks >> 2) * kQHalfBytes + (ks & 3) * 32, 16, 1024);
+#pragma unroll
+            for (int st = 0; st < kKvStages; ++st) {
+                k_desc0[st] = smem_desc(smem_u32(smem + kOffK + st * kTileBytes), 16, 1024);
+                v_desc0[st] = smem_desc(smem_u32(smem + kOffV + st * kTileBytes), kHalfBytes, 1024);
+            }
+            const uint64_t qx_desc = smem_desc_plain(smem_u32(smem + kOffQx), 128, kExtRowGroupBytes);
+            const uint64_t kp_desc = smem_desc_plain(smem_u32(smem + kOffKp), 128, kExtRowGroupBytes);
             bool ok = mbar_wait(q_full, 0, p.status);
             // O += P V for tile t: P (bf16 pairs, 8 columns per 16 keys) from tensor memory, V addressed MN-major:
             // 64-dim halves kHalfBytes apart (leading offset), groups of 8 keys 1 KiB apart (stride offset).
@@ -448,11 +467,12 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (!mbar_wait(&p_full[sb], (t >> 1) & 1, p.status)) return false;
                 if (!mbar_wait(&v_full[st], (t / kKvStages) & 1, p.status)) return false;
                 tc_fence_after();
-                const uint32_t v_addr = smem_u32(smem + kOffV + st * kTileBytes);
+                const uint64_t vd = st == 0 ? v_desc0[0] : v_desc0[kKvStages - 1];
+                const uint32_t p_tmem = tmem_base + kColS + sb * kTN;
+                umma_ts(tmem_base + kColO, p_tmem, vd, idesc_pv, t > 0);
 #pragma unroll
-                for (int kk = 0; kk < kTN / 16; ++kk)
-                    umma_ts(tmem_base + kColO, tmem_base + kColS + sb * kTN + kk * 8,
-                            smem_desc(v_addr + kk * 2048, kHalfBytes, 1024), idesc_pv, t > 0 || kk > 0);
+                for (int kk = 1; kk < kTN / 16; ++kk)
+                    umma_ts(tmem_base + kColO, p_tmem + kk * 8, desc_advance(vd, kk * 2048), idesc_pv, true);
                 tc_commit(&v_empty[st]);
                 return true;
             };
@@ -462,18 +482,14 @@ prefill_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (!ok) break;
                 tc_fence_after();
                 // S = Q K^T: both K-major, 16 dims (32 bytes) per step inside the 128-byte swizzled rows
-                const uint32_t k_addr = smem_u32(smem + kOffK + st * kTileBytes);
+                const uint64_t kd = st == 0 ? k_desc0[0] : k_desc0[kKvStages - 1];
+                const uint32_t s_tmem = tmem_base + kColS + sb * kTN;
                 if (dots) {
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        umma_ss(tmem_base + kColS + sb * kTN,
-                                smem_desc(q_addr + (ks >> 2) * kQHalfBytes + (ks & 3) * 32, 16, 1024),
-                                smem_desc(k_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024), idesc_qk, ks > 0);
-                    }
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        umma_ss(s_tmem, q_desc[ks], desc_advance(kd, (ks >> 2) * kHalfBytes + (ks & 3) * 32), idesc_qk, ks > 0);
                 }
-                if (alibi)
-                    umma_ss(tmem_base + kColS + sb * kTN, smem_desc_plain(smem_u32(smem + kOffQx), 128, kExtRowGroupBytes),
-                            smem_desc_plain(smem_u32(smem + kOffKp), 128, kExtRowGroupBytes), idesc_s, dots);
+                if (alibi) umma_ss(s_tmem, qx_desc, kp_desc, idesc_s, dots);
                 tc_commit(&s_full[sb]);
                 tc_commit(&k_empty[st]);
                 if (j >= 1) ok = issue_pv(j - 1);
