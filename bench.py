@@ -225,6 +225,13 @@ class DeviceBatch:
                 self.partial_out.data_ptr() if self.P else None, self.partial_lse.data_ptr() if self.P else None,
                 self.maxP, self.dt, stream)
 
+    def args_decode_single(self, i, stream):
+        """opt_gqa_paged_attention_decode as a single pass (what a one-launch step runs, minus the token store)."""
+        wl = self.wl
+        return (self.out.data_ptr(), self.q.data_ptr(), self.k_pools[i].data_ptr(), self.v_pools[i].data_ptr(),
+                self.tables.data_ptr(), wl.max_blocks, self.lens.data_ptr(), self.slopes.data_ptr(), wl.scale, wl.B,
+                wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, 0, None, None, 1, self.dt, stream)
+
     def args_reduce(self, stream):
         wl = self.wl
         if self.balanced:
@@ -460,12 +467,16 @@ def _step_fns(batch: DeviceBatch, stream):
     """Pre-marshalled foreign calls of one step, per pool copy."""
     sh = stream.cuda_stream
     lib, R, split = batch.lib, len(batch.k_pools), batch.P > 0
+    one_launch = step_launches(batch) == 1       # the library runs this step as a single pass: time that kernel
     a_app = [batch.args_append(i, sh) for i in range(R)]
-    a_dec = [batch.args_decode(i, sh) for i in range(R)]
+    a_dec = [batch.args_decode_single(i, sh) if one_launch else batch.args_decode(i, sh) for i in range(R)]
     a_step = [batch.args_step(i, sh) for i in range(R)]
+    split = split and not one_launch
     a_red = batch.args_reduce(sh) if split else None
     f_app = lib.opt_gqa_cache_append
-    if batch.balanced:
+    if one_launch:
+        f_dec, f_red = lib.opt_gqa_paged_attention_decode, None
+    elif batch.balanced:
         f_dec, f_red = lib.opt_gqa_paged_attention_decode_balanced, lib.opt_gqa_paged_attention_reduce_balanced
     else:
         f_dec, f_red = lib.opt_gqa_paged_attention_decode, lib.opt_gqa_paged_attention_reduce
@@ -821,7 +832,9 @@ def main():
     peak, peak_kind = measured_peak()
     alg = batch.algorithmic_bytes()
     achieved = alg / (dec["mean"] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (balanced split)" if batch.balanced else "decode_kernel",
+    roofline = {"bound": "hbm",
+                "kernel": "decode_tc_kernel (single pass)" if step_launches(batch) == 1 else
+                          "decode_stream_kernel (balanced split)" if batch.balanced else "decode_kernel",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(args.config),
                 "algorithmic_bytes_per_launch": alg, "kernel_us": dec["mean"] * 1e3,
@@ -866,7 +879,9 @@ def main():
             extra[w2.name] = {"tokens_per_s": w2.B * 1000 / (t_ms * 1e-3), "ms_per_step": t_ms / 1000,
                               "decode_us": d2["mean"] * 1e3, "decode_GBs": a2 / (d2["mean"] * 1e-3) / 1e9,
                               "frac_of_peak": a2 / (d2["mean"] * 1e-3) / 1e9 / peak, "partition_size": b2.P,
-                              "launches_timed": d2["launches"]}
+                              "launches_timed": d2["launches"], "launches_per_step": step_launches(b2),
+                              "decode_kernel": "decode_tc_kernel (single pass: the step is one launch)"
+                              if step_launches(b2) == 1 else "decode_stream_kernel (balanced split)"}
             del b2, w2
             torch.cuda.empty_cache()
         extra["other_decode_entry_points"] = entry_point_report(dev, peak)

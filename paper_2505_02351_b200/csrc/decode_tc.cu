@@ -22,11 +22,14 @@ namespace optgqa {
 namespace {
 
 // Warps per CTA (each with a private ring) and CTAs per SM the register budget is held to, for the two uses of the
-// kernel.  One CTA per (sequence, KV head) has the whole context to itself: eight warps, one CTA per SM.  One CTA per
-// (sequence, KV head, partition) has a few hundred tokens: two warps, six CTAs per SM, so that the CTA scheduler has
-// many small items to even out.  (Measured: single pass on 256 streams of 512-2048 tokens 35.3 us with 4 warps x 3
-// CTAs, 30.6 with 8 x 1; one partial per 512-token partition on long contexts 75.0 with 4 x 3, 71.8 with 2 x 6.)
-constexpr int kWarpsSingle = 8, kCtasSingle = 1;
+// kernel.  One CTA per (sequence, KV head) has the whole context to itself: twelve warps, one CTA per SM (192 KiB of
+// rings; measured on 256 streams of 512-2048 tokens: 8 warps 31.6 us, 10 30.7, 12 28.9, 13 32.2 and 14 31.4 -- past
+// twelve the register cap of 128 spills and the warps no longer divide over the four schedulers --, 6 warps x 2 CTAs
+// 32.5, 4 x 3 35.3; on 2048 ragged streams 218.7 with 8 warps, 204.8 with 12).  One CTA per (sequence, KV head,
+// partition) has a few hundred tokens: two warps, six CTAs per SM, so that the CTA scheduler has many small items to
+// even out (one partial per 512-token partition on long contexts: 1 warp x 12 CTAs 69.2 us, 2 x 6 68.7, 2 x 5 69.3,
+// 3 x 4 73.4, 4 x 3 75.7).
+constexpr int kWarpsSingle = 12, kCtasSingle = 1;
 constexpr int kWarpsSplit = 2, kCtasSplit = 6;
 constexpr int kTileTok = 16;                 // tokens per tile (one ring stage holds a K tile and a V tile)
 constexpr int kStages = 2;                   // ring depth per warp
