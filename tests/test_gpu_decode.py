@@ -453,3 +453,60 @@ def test_undersized_workspace_is_refused_before_anything_runs():
     torch.cuda.synchronize()
     assert bool((d.out == 3.0).all())
     assert torch.equal(d.k_cache.cpu(), wl.k_cache)        # the fused append did not run either
+
+
+def test_first_calls_from_several_host_threads_at_once():
+    """The per-device caches (symbol addresses, kernel attributes, SM count) are filled by whichever calls come
+    first; here four host threads of a fresh process make their first calls together, each on its own stream and
+    buffers, and every one must give the oracle's result."""
+    import subprocess
+    import sys
+    import textwrap
+
+    code = textwrap.dedent("""
+        import sys, threading
+        import numpy as np, torch
+        sys.path.insert(0, %r)
+        from paper_2505_02351_b200 import binding, workloads as W
+        from tests import util
+        binding.load()
+        torch.cuda.init()
+        wls = [W.make_custom("thr%%d" %% i, "bf16" if i %% 2 == 0 else "fp32", 8, 2, 128 if i < 2 else 64, 16,
+                             [700 + 37 * i, 33, 0, 260], seed=120 + i) for i in range(4)]
+        want = [util.oracle_attention(w) for w in wls]
+        devs = [util.DeviceWorkload(w) for w in wls]
+        streams = [torch.cuda.Stream() for _ in wls]
+        torch.cuda.synchronize()
+        barrier = threading.Barrier(len(wls))
+        errs = [None] * len(wls)
+
+        def work(i):
+            wl, d = wls[i], devs[i]
+            try:
+                barrier.wait()
+                with torch.cuda.stream(streams[i]):
+                    binding.cache_append(d.k_new, d.v_new, d.k_cache, d.v_cache, d.slot_mapping)
+                    if wl.dtype == "bf16":
+                        ws = torch.empty(binding.workspace_bytes(wl.B, wl.Hq, wl.D, 4), dtype=torch.uint8, device="cuda:0")
+                        binding.paged_attention_decode_balanced(d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+                                                                d.alibi_slopes, wl.scale, 256, ws, 4)
+                        binding.paged_attention_reduce_balanced(d.out, ws, d.context_lens, wl.Hkv, 256, 4)
+                    else:
+                        binding.paged_attention_decode(d.out, d.q, d.k_cache, d.v_cache, d.block_tables, d.context_lens,
+                                                       d.alibi_slopes, wl.scale)
+                streams[i].synchronize()
+                errs[i] = float(np.max(np.abs(d.out.double().cpu().numpy() - want[i])))
+            except Exception as e:          # noqa: BLE001
+                errs[i] = repr(e)
+
+        threads = [threading.Thread(target=work, args=(i,)) for i in range(len(wls))]
+        [t.start() for t in threads]
+        [t.join() for t in threads]
+        assert binding.device_status() == 0
+        for i, e in enumerate(errs):
+            assert isinstance(e, float) and e <= util.TOL[wls[i].dtype], (i, e)
+        print("threads ok", errs)
+    """ % util.ROOT)
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stdout + out.stderr
+    assert "threads ok" in out.stdout

@@ -1,4 +1,6 @@
 """Helpers shared by the parity tests: run a workload through the CUDA library and through the oracle."""
+import os
+
 import numpy as np
 import torch
 
@@ -6,6 +8,7 @@ import oracle
 from paper_2505_02351_b200 import binding
 from paper_2505_02351_b200 import workloads as W
 
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))   # the repository root (for child processes)
 TOL = {"fp32": 1e-5, "bf16": 2e-2}   # max-abs tolerance on attention outputs (fp32 accumulation)
 
 
