@@ -392,6 +392,10 @@ extern "C++" {
 template <typename V>
 __global__ void __launch_bounds__(256) gather_host_kernel(const HostGather g) {
     const unsigned tid = blockIdx.x * blockDim.x + threadIdx.x, nthreads = gridDim.x * blockDim.x, total = g.first[6];
+    // The words are requested from the host before the wait for the preceding kernel of the stream (the bus round
+    // trip overlaps that kernel's tail); they are stored only after it, since that kernel may still read the staging
+    // buffers.  This kernel never lets its own dependents start early: they read what it writes before their wait.
+    bool waited = false;
     for (unsigned base = tid; base < total; base += 4 * nthreads) {
         V v[4];
         int arr[4];
@@ -407,12 +411,17 @@ __global__ void __launch_bounds__(256) gather_host_kernel(const HostGather g) {
                 v[u] = static_cast<const V*>(g.src[a])[i - g.first[a]];
             }
         }
+        if (!waited) {
+            grid_dependency_wait();
+            waited = true;
+        }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const unsigned i = base + u * nthreads;
             if (arr[u] >= 0) static_cast<V*>(g.dst[arr[u]])[i - g.first[arr[u]]] = v[u];
         }
     }
+    if (!waited) grid_dependency_wait();
 }
 }  // extern "C++"
 
@@ -510,9 +519,9 @@ static int host_step(void* out_host, const void* q_host, const void* k_new_host,
     if (kResolved && !pinned) return OPT_GQA_ERR_ALIGN;     // views must be 4-byte aligned, the one of out 16-byte
     if (pinned) {
         const unsigned ctas = (unsigned)((words + 255) / 256 < 148 ? (words + 255) / 256 : 148);
-        if (wide) gather_host_kernel<uint4><<<ctas, 256, 0, cs>>>(g);
-        else gather_host_kernel<uint32_t><<<ctas, 256, 0, cs>>>(g);
-        if (cudaGetLastError() != cudaSuccess) return OPT_GQA_ERR_CUDA;
+        const int rc = wide ? launch_dependent(gather_host_kernel<uint4>, dim3(ctas), dim3(256), 0, cs, g)
+                            : launch_dependent(gather_host_kernel<uint32_t>, dim3(ctas), dim3(256), 0, cs, g);
+        if (rc != OPT_GQA_OK) return rc;
     } else {
         bool ok = true;
         for (int a = 0; a < 6; ++a)
