@@ -54,8 +54,11 @@ __device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
 }
 
 // 128 + code for the two codes in nibbles `shift/4` and `shift/4 + 4` of w, as a bf16 pair.
+// (One three-input logic instruction: (a & mask) | magic.  Written out because the compiler otherwise spends two.)
 __device__ __forceinline__ uint32_t codes_to_bf16x2(uint32_t w, int shift) {
-    return ((w >> shift) & 0x000F000Fu) | 0x43004300u;
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(w >> shift), "r"(0x000F000Fu), "r"(0x43004300u));
+    return d;
 }
 
 __device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
