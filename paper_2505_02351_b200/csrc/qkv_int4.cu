@@ -45,6 +45,7 @@ struct ProjParams {
     const int64_t* slot_mapping;
     int T, K, N, Hq, Hkv, D, bs;
     long long num_blocks;
+    int whole_ctas;          // CTAs 0 .. whole_ctas - 1 take a tile each; the rest share the remaining tiles, a cluster per tile
 };
 
 __device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
@@ -65,26 +66,86 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
     return __bfloat16_as_ushort(__float2bfloat16_rn(f));
 }
 
+// Rounds the sums of features n, n + 1 of token t to bf16 and stores them where they belong: the query output, the
+// plain key/value outputs, the paged cache at the token's slot.
+__device__ __forceinline__ void store_pair(const ProjParams& p, int t, int n, float s0, float s1) {
+    const uint32_t pair = (uint32_t)float_to_bf16_bits(s0) | ((uint32_t)float_to_bf16_bits(s1) << 16);
+    const int qn = p.Hq * p.D, kvn = p.Hkv * p.D;
+    if (n < qn) {
+        *reinterpret_cast<uint32_t*>(p.q_out + (size_t)t * qn + n) = pair;
+        return;
+    }
+    const bool is_k = n < qn + kvn;
+    const int col = n - qn - (is_k ? 0 : kvn);
+    uint16_t* plain = is_k ? p.k_out : p.v_out;
+    uint16_t* cache = is_k ? p.k_cache : p.v_cache;
+    if (plain) *reinterpret_cast<uint32_t*>(plain + (size_t)t * kvn + col) = pair;
+    if (cache) {
+        const long long slot = p.slot_mapping[t];
+        const long long page = slot / p.bs;
+        if (slot >= 0 && page < p.num_blocks) {
+            const int h = col / p.D, d = col % p.D;
+            const size_t dst = (((size_t)page * p.Hkv + h) * p.bs + (size_t)(slot % p.bs)) * p.D + d;
+            *reinterpret_cast<uint32_t*>(cache + dst) = pair;
+        }
+    }
+}
+
+// Thread-block cluster: this CTA's rank and the cluster's size, the cluster-wide barrier, and a read of the same
+// shared-memory location in another CTA of the cluster.
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float2 ld_cluster_float2(const void* local_smem, uint32_t rank) {
+    uint32_t remote;
+    float2 v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem)), "r"(rank));
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(remote) : "memory");
+    return v;
+}
+
 // NT: token tiles of eight per CTA; CPG: 64-row chunks per quantisation group.
+//
+// One CTA per 32-feature tile leaves a last, short wave: N / 32 tiles rarely divide by the CTAs the GPU holds, and a
+// tile's CTA is a chain of K / 64 / 8 chunks per warp whatever else runs.  The launch therefore gives whole tiles only
+// to as many CTAs as fill complete waves (p.whole_ctas); each remaining tile goes to a cluster whose CTAs take a
+// slice of K each, so that the tail is a fraction as long, and add their partial sums up through distributed shared
+// memory (rank order, so the result does not depend on timing).
 template <int NT, int CPG>
 __global__ void __launch_bounds__(kProjWarps * 32, 2) qkv_int4_kernel(const ProjParams p) {
     constexpr int PF = NT == 1 ? 4 : 2;   // chunks in flight per warp; a multiple of CPG
     static_assert(PF % CPG == 0, "ring must hold whole groups");
     constexpr int GSLOTS = PF / CPG;
     __shared__ float red[kProjWarps][8 * NT][kRedStride];
+    __shared__ __align__(8) float cta_sum[8 * NT][kRedStride];       // a K slice's sums, read by the cluster
 
     grid_dependency_launch();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int r = lane >> 2, c = lane & 3;
     const int KC = p.K >> 6;
-    const int groups = KC / CPG;
+    // the CTA's tile and its slice of the tile's quantisation groups; the warps split the slice
+    const bool sliced = (int)blockIdx.x >= p.whole_ctas;
+    const int csize = sliced ? (int)cluster_size() : 1, crank = sliced ? (int)cluster_rank() : 0;
+    const int tile = sliced ? p.whole_ctas + ((int)blockIdx.x - p.whole_ctas) / csize : (int)blockIdx.x;
+    const int tile_groups = KC / CPG;
+    const int g0 = tile_groups * crank / csize, groups = tile_groups * (crank + 1) / csize - g0;
     const int gpw = (groups + kProjWarps - 1) / kProjWarps;
-    const int kc0 = min(groups, warp * gpw) * CPG;
-    const int kc1 = min(groups, (warp + 1) * gpw) * CPG;
-    const int n0 = blockIdx.x * kFeatPerCta;
+    const int kc0 = (g0 + min(groups, warp * gpw)) * CPG;
+    const int kc1 = (g0 + min(groups, (warp + 1) * gpw)) * CPG;
+    const int n0 = tile * kFeatPerCta;
     const int t0 = blockIdx.y * 8 * NT;
 
-    const uint4* w0 = p.wp + (size_t)(2 * blockIdx.x) * KC * 32 + lane;
+    const uint4* w0 = p.wp + (size_t)(2 * tile) * KC * 32 + lane;
     const uint4* w1 = w0 + (size_t)KC * 32;
     const uint4* xrow[NT];
 #pragma unroll
@@ -198,39 +259,35 @@ __global__ void __launch_bounds__(kProjWarps * 32, 2) qkv_int4_kernel(const Proj
 
     // one thread per (token, pair of features): 16 pairs x 8 NT tokens
     static_assert(16 * 8 * NT <= kProjWarps * 32, "the epilogue needs a thread per output pair");
+    const int tl = threadIdx.x >> 4, f = (threadIdx.x & 15) * 2;
+    float s0 = 0.f, s1 = 0.f;
     if (threadIdx.x < 16 * 8 * NT) {
-        const int tl = threadIdx.x >> 4, f = (threadIdx.x & 15) * 2;
-        const int t = t0 + tl;
-        if (t < p.T) {
-            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-            for (int w = 0; w < kProjWarps; ++w) {
-                s0 += red[w][tl][f];
-                s1 += red[w][tl][f + 1];
-            }
-            const uint32_t pair = (uint32_t)float_to_bf16_bits(s0) | ((uint32_t)float_to_bf16_bits(s1) << 16);
-            const int n = n0 + f;
-            const int qn = p.Hq * p.D, kvn = p.Hkv * p.D;
-            if (n < qn) {
-                *reinterpret_cast<uint32_t*>(p.q_out + (size_t)t * qn + n) = pair;
-            } else {
-                const bool is_k = n < qn + kvn;
-                const int col = n - qn - (is_k ? 0 : kvn);
-                uint16_t* plain = is_k ? p.k_out : p.v_out;
-                uint16_t* cache = is_k ? p.k_cache : p.v_cache;
-                if (plain) *reinterpret_cast<uint32_t*>(plain + (size_t)t * kvn + col) = pair;
-                if (cache) {
-                    const long long slot = p.slot_mapping[t];
-                    const long long page = slot / p.bs;
-                    if (slot >= 0 && page < p.num_blocks) {
-                        const int h = col / p.D, d = col % p.D;
-                        const size_t dst = (((size_t)page * p.Hkv + h) * p.bs + (size_t)(slot % p.bs)) * p.D + d;
-                        *reinterpret_cast<uint32_t*>(cache + dst) = pair;
-                    }
-                }
-            }
+        for (int w = 0; w < kProjWarps; ++w) {
+            s0 += red[w][tl][f];
+            s1 += red[w][tl][f + 1];
         }
     }
+    if (!sliced) {
+        if (threadIdx.x < 16 * 8 * NT && t0 + tl < p.T) store_pair(p, t0 + tl, n0 + f, s0, s1);
+        return;
+    }
+    // a K slice: the cluster's CTAs exchange their sums; CTA `crank` finishes an equal share of the outputs
+    if (threadIdx.x < 16 * 8 * NT) *reinterpret_cast<float2*>(&cta_sum[tl][f]) = make_float2(s0, s1);
+    cluster_sync_all();
+    const int share = 16 * 8 * NT / csize;
+    if ((int)threadIdx.x < share) {
+        const int idx = crank * share + threadIdx.x;
+        const int tk = idx >> 4, fk = (idx & 15) * 2;
+        float t_0 = 0.f, t_1 = 0.f;
+        for (int k = 0; k < csize; ++k) {
+            const float2 v = ld_cluster_float2(&cta_sum[tk][fk], (uint32_t)k);
+            t_0 += v.x;
+            t_1 += v.y;
+        }
+        if (t0 + tk < p.T) store_pair(p, t0 + tk, n0 + fk, t_0, t_1);
+    }
+    cluster_sync_all();           // no CTA's shared memory goes away while another still reads it
 }
 
 // One thread per uint4 of wp, and (second part of the grid-stride range) one per entry of sz.
@@ -271,6 +328,53 @@ int4_prepack_kernel(uint4* __restrict__ wp, uint32_t* __restrict__ sz, const uin
         // bf16 of 128 + zero: 0x4300 with the zero point in the low mantissa bits
         sz[e] = (uint32_t)scales[e] | ((0x4300u | zero) << 16);
     }
+}
+
+constexpr int kSliceCtas = 4;         // CTAs of a cluster: K slices of a tail tile
+
+// Launches the projection for `tiles` feature tiles and `chunks` passes over the tokens.  With one pass, the tiles
+// beyond the last complete wave of CTAs (as many clusters as the GPU holds at once) are cut into kSliceCtas slices of
+// K each, unless they are more than half a wave: then, or when the slices would not hold a group each, every tile
+// keeps its own CTA.
+template <int NT, int CPG>
+int launch_proj(ProjParams p, int tiles, int chunks, cudaStream_t stream) {
+    static std::atomic<int> wave_ctas[kMaxDevices];       // 0: not asked yet
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kProjWarps * 32);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = kSliceCtas;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+
+    int wave = 0, dev = 0;
+    if (chunks == 1 && (p.K >> 6) / CPG >= kSliceCtas && cudaGetDevice(&dev) == cudaSuccess) {
+        const bool cached = dev >= 0 && dev < kMaxDevices;
+        wave = cached ? wave_ctas[dev].load(std::memory_order_acquire) : 0;
+        if (wave == 0) {
+            cfg.gridDim = dim3(kSliceCtas);
+            cfg.numAttrs = 2;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, qkv_int4_kernel<NT, CPG>, &cfg) != cudaSuccess) clusters = 0;
+            wave = clusters > 0 ? clusters * kSliceCtas : -1;
+            if (cached) wave_ctas[dev].store(wave, std::memory_order_release);
+        }
+    }
+    const int tail = wave > 0 ? tiles % wave : 0;
+    if (tail > 0 && tiles > wave && 2 * tail <= wave) {
+        p.whole_ctas = tiles - tail;
+        cfg.gridDim = dim3((unsigned)(p.whole_ctas + tail * kSliceCtas), (unsigned)chunks);
+        cfg.numAttrs = 2;
+    } else {
+        p.whole_ctas = tiles;
+        cfg.gridDim = dim3((unsigned)tiles, (unsigned)chunks);
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, qkv_int4_kernel<NT, CPG>, p) == cudaSuccess ? OPT_GQA_OK : OPT_GQA_ERR_CUDA;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -336,10 +440,7 @@ extern "C" int opt_gqa_qkv_project_int4(void* q_out, void* k_out, void* v_out, v
     const int NT = T <= 8 ? 1 : 2;
     const long long chunks = ((long long)T + 8 * NT - 1) / (8 * NT);
     if (chunks > 65535) return OPT_GQA_ERR_SHAPE;
-    dim3 grid((unsigned)(Nl / kFeatPerCta), (unsigned)chunks), block(kProjWarps * 32);
-    if (NT == 1)
-        return gs == 64 ? launch_dependent(qkv_int4_kernel<1, 1>, grid, block, 0, cs, p)
-                        : launch_dependent(qkv_int4_kernel<1, 2>, grid, block, 0, cs, p);
-    return gs == 64 ? launch_dependent(qkv_int4_kernel<2, 1>, grid, block, 0, cs, p)
-                    : launch_dependent(qkv_int4_kernel<2, 2>, grid, block, 0, cs, p);
+    const int tiles = (int)(Nl / kFeatPerCta);
+    if (NT == 1) return gs == 64 ? launch_proj<1, 1>(p, tiles, (int)chunks, cs) : launch_proj<1, 2>(p, tiles, (int)chunks, cs);
+    return gs == 64 ? launch_proj<2, 1>(p, tiles, (int)chunks, cs) : launch_proj<2, 2>(p, tiles, (int)chunks, cs);
 }

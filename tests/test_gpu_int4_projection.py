@@ -92,6 +92,13 @@ def test_projection_70b_like_shape():
     _run(3, 8, 64, 8, 128, 8192, 128, bs=32)
 
 
+@pytest.mark.parametrize("T,gs,K", [(5, 128, 1024), (16, 64, 512), (8, 128, 640)])
+def test_projection_more_tiles_than_one_wave_of_ctas(T, gs, K):
+    """N / 32 = 320 tiles exceed what a B200 holds at once: the tiles past the last complete wave are cut into K slices
+    whose CTAs add their sums up across a cluster (K = 640 with 128-row groups gives slices of unequal length)."""
+    _run(40 + T, T, 64, 8, 128, K, gs, bs=32)
+
+
 def test_projection_rejects_bad_arguments():
     lib = binding.load()
     x = torch.zeros((8, 512), dtype=torch.bfloat16, device=DEV)
