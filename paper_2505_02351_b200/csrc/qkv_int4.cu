@@ -3,7 +3,8 @@
 // values written straight into the paged cache (Algorithm 1, "Reshape and store K, V into C_K, C_V").
 //
 // The step is a matrix-vector product per token: every weight is read once and used T times, so for the
-// few tokens of a decode step the kernel is bound by the HBM read of the codes (half a byte per weight).
+// few tokens of a decode step the floor is the HBM read of the codes (half a byte per weight); what the
+// kernel has to keep small to get near it is the integer work of turning codes into bf16.
 // The product runs on the tensor cores all the same, because unpacking eight codes and multiplying them
 // with T activations each on the plain ALUs would cost more issue slots than the memory system leaves:
 // the output features are the rows of an m16n8k16 tile, the tokens its eight columns, and the codes go
