@@ -92,11 +92,14 @@ def test_projection_70b_like_shape():
     _run(3, 8, 64, 8, 128, 8192, 128, bs=32)
 
 
-@pytest.mark.parametrize("T,gs,K", [(5, 128, 1024), (16, 64, 512), (8, 128, 640)])
-def test_projection_more_tiles_than_one_wave_of_ctas(T, gs, K):
-    """N / 32 = 320 tiles exceed what a B200 holds at once: the tiles past the last complete wave are cut into K slices
-    whose CTAs add their sums up across a cluster (K = 640 with 128-row groups gives slices of unequal length)."""
-    _run(40 + T, T, 64, 8, 128, K, gs, bs=32)
+@pytest.mark.parametrize("T,gs,K,Hq", [(5, 128, 1024, 64), (16, 64, 512, 64), (8, 128, 640, 64), (3, 64, 256, 80),
+                                        (11, 128, 512, 96), (8, 64, 192, 64)])
+def test_projection_more_tiles_than_one_wave_of_ctas(T, gs, K, Hq):
+    """N / 32 = 320 tiles (Hq 64), 384 (Hq 80) or 448 (Hq 96) exceed what a B200 holds at once: the tiles past the
+    last complete wave are cut into K slices whose CTAs add their sums up across a cluster, unless they are more than
+    half a wave (Hq 96) or there are fewer groups than slices (K 192, gs 64: three).  K = 640 with 128-row groups gives
+    slices of unequal length."""
+    _run(40 + T, T, Hq, 8, 128, K, gs, bs=32)
 
 
 def test_projection_rejects_bad_arguments():
