@@ -33,6 +33,7 @@ namespace {
 constexpr int kProjWarps = 8;         // warps of a CTA; they split K between them
 constexpr int kFeatPerCta = 32;       // output features of a CTA: two m16 tiles
 constexpr int kRedStride = 36;        // floats between the tokens' rows of the cross-warp sum (bank spread)
+constexpr int kMaxSlices = 4;         // CTAs of a cluster that share a tile, a slice of K each
 
 struct ProjParams {
     const uint16_t* x;       // [T, K] bf16
@@ -92,7 +93,7 @@ __device__ __forceinline__ void store_pair(const ProjParams& p, int t, int n, fl
     }
 }
 
-// Thread-block cluster: this CTA's rank and the cluster's size, the cluster-wide barrier, and a read of the same
+// Thread-block cluster: this CTA's rank and the cluster's size, the cluster-wide barrier, and a store to the same
 // shared-memory location in another CTA of the cluster.
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
@@ -107,12 +108,10 @@ __device__ __forceinline__ uint32_t cluster_size() {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ float2 ld_cluster_float2(const void* local_smem, uint32_t rank) {
+__device__ __forceinline__ void st_cluster_float2(const void* local_smem, uint32_t rank, float2 v) {
     uint32_t remote;
-    float2 v;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem)), "r"(rank));
-    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(remote) : "memory");
-    return v;
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote), "f"(v.x), "f"(v.y) : "memory");
 }
 
 // NT: token tiles of eight per CTA; CPG: 64-row chunks per quantisation group.
@@ -128,7 +127,7 @@ __global__ void __launch_bounds__(kProjWarps * 32, 2) qkv_int4_kernel(const Proj
     static_assert(PF % CPG == 0, "ring must hold whole groups");
     constexpr int GSLOTS = PF / CPG;
     __shared__ float red[kProjWarps][8 * NT][kRedStride];
-    __shared__ __align__(8) float cta_sum[8 * NT][kRedStride];       // a K slice's sums, read by the cluster
+    __shared__ __align__(8) float recv[kMaxSlices][8 * NT][kRedStride];   // K slices' sums, written by the cluster's CTAs
 
     grid_dependency_launch();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -273,22 +272,24 @@ __global__ void __launch_bounds__(kProjWarps * 32, 2) qkv_int4_kernel(const Proj
         if (threadIdx.x < 16 * 8 * NT && t0 + tl < p.T) store_pair(p, t0 + tl, n0 + f, s0, s1);
         return;
     }
-    // a K slice: the cluster's CTAs exchange their sums; CTA `crank` finishes an equal share of the outputs
-    if (threadIdx.x < 16 * 8 * NT) *reinterpret_cast<float2*>(&cta_sum[tl][f]) = make_float2(s0, s1);
-    cluster_sync_all();
+    // a K slice: CTA o of the cluster finishes an equal share of the outputs; every CTA writes its sums for that
+    // share into slot `crank` of o's shared memory, and after one cluster barrier each CTA adds up what it received,
+    // in rank order.  (Nothing touches another CTA's shared memory after the barrier, so a CTA may end at once.)
     const int share = 16 * 8 * NT / csize;
+    if (threadIdx.x < 16 * 8 * NT)
+        st_cluster_float2(&recv[crank][tl][f], (uint32_t)(threadIdx.x / share), make_float2(s0, s1));
+    cluster_sync_all();
     if ((int)threadIdx.x < share) {
         const int idx = crank * share + threadIdx.x;
         const int tk = idx >> 4, fk = (idx & 15) * 2;
         float t_0 = 0.f, t_1 = 0.f;
         for (int k = 0; k < csize; ++k) {
-            const float2 v = ld_cluster_float2(&cta_sum[tk][fk], (uint32_t)k);
+            const float2 v = *reinterpret_cast<const float2*>(&recv[k][tk][fk]);
             t_0 += v.x;
             t_1 += v.y;
         }
         if (t0 + tk < p.T) store_pair(p, t0 + tk, n0 + fk, t_0, t_1);
     }
-    cluster_sync_all();           // no CTA's shared memory goes away while another still reads it
 }
 
 // One thread per uint4 of wp, and (second part of the grid-stride range) one per entry of sz.
@@ -331,7 +332,7 @@ int4_prepack_kernel(uint4* __restrict__ wp, uint32_t* __restrict__ sz, const uin
     }
 }
 
-constexpr int kSliceCtas = 4;         // CTAs of a cluster: K slices of a tail tile
+constexpr int kSliceCtas = kMaxSlices;        // CTAs of a cluster: K slices of a tail tile
 
 // Launches the projection for `tiles` feature tiles and `chunks` passes over the tokens.  With one pass, the tiles
 // beyond the last complete wave of CTAs (as many clusters as the GPU holds at once) are cut into kSliceCtas slices of
