@@ -102,6 +102,21 @@ def test_projection_more_tiles_than_one_wave_of_ctas(T, gs, K, Hq):
     _run(40 + T, T, Hq, 8, 128, K, gs, bs=32)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_projection_random_shapes(seed):
+    """Drawn token counts (one pass of 8, of 16, several passes), group sizes, widths that are odd multiples of a
+    group, head counts and destinations."""
+    rng = np.random.default_rng(3000 + seed)
+    T = int(rng.choice([1, 2, 7, 8, 9, 15, 16, 17, 33]))
+    gs = int(rng.choice([64, 128]))
+    K = gs * int(rng.integers(1, 13))
+    D = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    Hq = Hkv * int(rng.choice([1, 2, 4, 8]))
+    plain, cache = [(True, True), (True, False), (False, True)][int(rng.integers(0, 3))]
+    _run(3100 + seed, T, Hq, Hkv, D, K, gs, bs=int(rng.choice([16, 32])), plain=plain, cache=cache)
+
+
 def test_projection_rejects_bad_arguments():
     lib = binding.load()
     x = torch.zeros((8, 512), dtype=torch.bfloat16, device=DEV)
