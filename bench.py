@@ -836,15 +836,19 @@ def main():
         e2e_s, h2d, d2h, pipe_s = run_e2e(batch, E2E_STEPS, 10)
         e2e_s = max_over_ranks(e2e_s, str(dev))
         pipe_s = max_over_ranks(pipe_s, str(dev))
-        e2e = {"value": tokens_all * E2E_STEPS / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": E2E_STEPS, "us_per_step": e2e_s / E2E_STEPS * 1e6,
-               "api": "opt_gqa_decode_step_mapped (pinned host q/k_new/v_new/slots/tables/lens in, out back, "
-                      "stream synchronised per step)"}
+        # The end-to-end figure is the loop a serving host runs: every step brings its inputs in from pinned host
+        # memory and stores its result to the host, and the host enqueues step i + 1 before it waits for (and reads)
+        # step i's result.  The same steps with the host blocking after every call are reported beside it.
+        e2e = {"value": tokens_all * E2E_STEPS / pipe_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": E2E_STEPS, "us_per_step": pipe_s / E2E_STEPS * 1e6,
+               "api": "opt_gqa_decode_step_mapped (pinned host q/k_new/v_new/slots/tables/lens in, out back to the "
+                      "host; step i + 1 is enqueued before the host waits for step i's result and reads it)"}
         e2e["frac_of_value"] = e2e["value"] / value
-        e2e["host_one_step_ahead"] = {
-            "value": tokens_all * E2E_STEPS / pipe_s, "us_per_step": pipe_s / E2E_STEPS * 1e6,
-            "frac_of_value": tokens_all * E2E_STEPS / pipe_s / value,
-            "what": "the same call and transfers, step i + 1 enqueued before the host waits for step i's result"}
+        e2e["synchronised_per_step"] = {
+            "value": tokens_all * E2E_STEPS / e2e_s, "us_per_step": e2e_s / E2E_STEPS * 1e6,
+            "frac_of_value": tokens_all * E2E_STEPS / e2e_s / value,
+            "what": "the same call and transfers with the stream synchronised after every call (the host idle "
+                    "while the step runs, the GPU idle while the host launches)"}
         ceiling = read_only_ceiling(dev, torch.cuda.current_stream())
     clocks = sampler.stop()
     status = binding.device_status()
