@@ -454,6 +454,101 @@ def entry_point_report(dev, peak) -> dict:
     return out
 
 
+def masked_entry_point_report(dev, peak) -> dict:
+    """Side measurement of the entry points for the other masks of Algorithm 1: the prompt branch over contiguous
+    k, v (empty caches), the local window in decode (cfg 3 shapes, 4096-token window) and in chunked prefill (cfg 5
+    shapes, 1024-token window).  Back-to-back calls, CUDA events around the run; the decode rotates pool copies."""
+    import numpy as np
+    import torch
+
+    from paper_2505_02351_b200 import binding
+    from paper_2505_02351_b200 import workloads as W
+
+    lib = binding.load()
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+    sustained, burst, kind = measured_tensor_peak()
+    out = {}
+
+    def timed(call, n, warm=5):
+        for i in range(warm):
+            call(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(n):
+            call(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / n            # us per call
+
+    # ---- prompt branch, empty caches: 4 prompts of 4096 tokens, 32 query / 8 KV heads of 128, bf16
+    B, n, Hq, Hkv, D = 4, 4096, 32, 8, 128
+    gen = torch.Generator().manual_seed(17)
+    mk = lambda *shape: torch.randn(shape, generator=gen).to(torch.bfloat16).to(dev)
+    q, k, v = mk(B * n, Hq, D), mk(B * n, Hkv, D), mk(B * n, Hkv, D)
+    o = torch.empty_like(q)
+    qsl = torch.arange(0, (B + 1) * n, n, dtype=torch.int32, device=dev)
+    slopes = torch.tensor([2.0 ** (-8.0 * (h + 1) / Hq) for h in range(Hq)], dtype=torch.float32, device=dev)
+    a = (o.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(), qsl.data_ptr(), B * n, n, slopes.data_ptr(),
+         1.0 / float(np.sqrt(D)), B, Hq, Hkv, D, 1, sh)
+    us = timed(lambda i: check(lib.opt_gqa_prompt_attention(*a), "prompt_attention"), 20)
+    flop = 4.0 * D * Hq * B * (n * (n + 1) // 2)
+    tf = flop / us / 1e6
+    out["prompt_attention_4x4096"] = {"us_per_call": us, "TFLOPs": tf, "frac_of_bf16_peak": tf / sustained,
+                                      "peak_kind": f"of {kind} (sustained cuBLAS bf16)", "flop_per_call": flop,
+                                      "bound": "tensor"}
+    del q, k, v, o
+
+    # ---- decode with a local window on the long-sequence workload
+    wl = W.make_config(3)
+    window, P = 4096, 512
+    b = DeviceBatch(wl, P, COPIES, dev)
+    lens = wl.context_lens.numpy().astype("int64")
+    es = 2
+    alg = int(np.minimum(lens, window).sum()) * 2 * wl.Hkv * wl.D * es + 2 * wl.B * wl.Hq * wl.D * es
+    a_loc = [(b.out.data_ptr(), b.q.data_ptr(), b.k_pools[i].data_ptr(), b.v_pools[i].data_ptr(), b.tables.data_ptr(),
+              wl.max_blocks, b.lens.data_ptr(), b.slopes.data_ptr(), wl.scale, wl.B, wl.Hq, wl.Hkv, wl.D, wl.bs,
+              wl.num_blocks, P, b.workspace.data_ptr(), b.ws_bytes, b.maxP, window, b.dt, sh)
+             for i in range(len(b.k_pools))]
+    R = len(a_loc)
+    us = timed(lambda i: check(lib.opt_gqa_paged_attention_decode_local(*a_loc[i % R]), "decode_local"), 200, 20)
+    out["decode_local_window_4096_cfg3"] = {"us_per_call": us, "GBs": alg / us / 1e3, "frac_of_peak": alg / us / 1e3 / peak,
+                                            "algorithmic_bytes_per_call": alg, "bound": "hbm",
+                                            "note": "two launches (split decode over the windows, merge); 67 MB per "
+                                                    "call, pool copies rotated"}
+    del b
+    torch.cuda.empty_cache()
+
+    # ---- chunked prefill with a local window
+    wl = W.make_config(5)
+    pb = PrefillBatch(wl, dev)
+    window = 1024
+    qsl_h = wl.q_start_loc.numpy().astype("int64")
+    nn = wl.context_lens.numpy().astype("int64")
+    pairs = 0
+    for s in range(wl.B):
+        ql = int(qsl_h[s + 1] - qsl_h[s])
+        pos = np.arange(int(nn[s]) - ql, int(nn[s]), dtype=np.int64)
+        pairs += int(np.minimum(pos + 1, window).sum())
+    flop = 4.0 * wl.D * wl.Hq * pairs
+    check(lib.opt_gqa_cache_append(pb.k_new.data_ptr(), pb.v_new.data_ptr(), pb.k_pool.data_ptr(), pb.v_pool.data_ptr(),
+                                   pb.slots.data_ptr(), wl.T, wl.Hkv, wl.D, wl.bs, wl.num_blocks, 1, sh), "cache_append")
+    a_pl = (pb.out.data_ptr(), pb.q.data_ptr(), pb.qsl.data_ptr(), wl.T, pb.max_q_len, pb.k_pool.data_ptr(),
+            pb.v_pool.data_ptr(), pb.tables.data_ptr(), wl.max_blocks, pb.lens.data_ptr(), pb.slopes.data_ptr(), wl.scale,
+            wl.B, wl.Hq, wl.Hkv, wl.D, wl.bs, wl.num_blocks, window, 1, sh)
+    us = timed(lambda i: check(lib.opt_gqa_paged_attention_prefill_local(*a_pl), "prefill_local"), 20)
+    tf = flop / us / 1e6
+    out["prefill_local_window_1024_cfg5"] = {"us_per_call": us, "TFLOPs": tf, "frac_of_bf16_peak": tf / sustained,
+                                             "peak_kind": f"of {kind} (sustained cuBLAS bf16)", "flop_per_call": flop,
+                                             "bound": "tensor",
+                                             "note": "flop counted over the (token, key) pairs inside the window; the "
+                                                     "tiles that straddle its edges are multiplied whole"}
+    del pb
+    torch.cuda.empty_cache()
+    return out
+
+
 def check(rc: int, what: str):
     if rc != 0:
         raise RuntimeError(f"{what} failed with status {rc}")
@@ -912,6 +1007,7 @@ def main():
             torch.cuda.empty_cache()
         extra["other_decode_entry_points"] = entry_point_report(dev, peak)
         extra[W.CONFIG_NAMES[5]] = prefill_report(dev, 20, 3)
+        extra["other_masks"] = masked_entry_point_report(dev, peak)
         extra["int4_qkv_projection"] = projection_report(dev)
         line["other_workloads"] = extra
         line["cpu_baseline"] = cpu_baseline(wl)
